@@ -1,0 +1,188 @@
+/*
+ * libsste -- the S-STE 2:4 sparse-training linear layer for NVIDIA B200 (sm_100a).
+ *
+ * One training iteration of an S-STE linear (Sec. 2: prune, run forward/backward
+ * with the sparse weight, update the dense weight) maps onto these calls:
+ *
+ *   step 0 only   sste_beta_init          beta = <w,S_soft(w)> / ||S_soft(w)||^2      (Eq. 5)
+ *   every step    sste_project_compress   w~ = beta * S_soft(w), 2:4 values + metadata (Eq. 4, Sec. 4.2)
+ *                 sste_linear_fwd         Z = X w~^T            sparse tensor cores   (Sec. 5.1)
+ *                 sste_mvue_sparsify      MVUE(grad_Z^T)        2:4 along tokens      (Sec. 5.1)
+ *                 sste_linear_bwd_weight  grad_W = MVUE(grad_Z^T) X   sparse          (Sec. 5.1)
+ *                 sste_linear_bwd_input   grad_X = grad_Z w~          dense           (Sec. 5.1)
+ *   FP8 variant   sste_amax, sste_fp8_scale, sste_quantize_fp8 + the E4M3/E5M2 dtypes (Sec. 5.2)
+ *
+ * Conventions (all entry points)
+ *   - Every tensor pointer is DEVICE memory owned by the caller, row-major and
+ *     contiguous.  The library allocates no tensor memory and keeps no pointer
+ *     after a call returns.  Scalars beta / scales are DEVICE pointers to one
+ *     float so that no call needs a host synchronisation.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it.
+ *   - O = out features, I = in features, T = tokens.  O, I and T must be
+ *     multiples of 128 and tensor pointers 128-byte aligned, otherwise
+ *     SSTE_ERR_SHAPE / SSTE_ERR_ALIGN is returned BEFORE anything is launched.
+ *   - A device that is not compute capability 10.x gives SSTE_ERR_ARCH.  There
+ *     is no CPU or other fallback.
+ *   - Kernels never trap.  Bounded waits that expire record SSTE_ERR_TIMEOUT
+ *     in the context's device status word, read by sste_poll_device_status.
+ *   - bf16 tensors hold IEEE bfloat16 bit patterns, E4M3 is the "fn" flavour
+ *     (max 448, no infinity), E5M2 is IEEE-like (max finite 57344).
+ *
+ * Compressed 2:4 operand ("vals" + "meta") of a logical [rows, K] matrix whose
+ * groups of four run along K:
+ *   vals  [rows, K/2]  the two kept values of every group, ascending position, row-major.
+ *   meta  one 4-bit code per group: p0 | (p1 << 2), p0 < p1 the kept positions.  Codes are
+ *         stored in the image the sparse tensor-core instruction reads from tensor memory,
+ *         as 2 KB atoms of 128 rows x 128 logical K, atom (rb, kb) at byte
+ *         (rb * (K/128) + kb) * 2048.  Inside an atom, row m and K-offset k (group k/4):
+ *           16-bit operands:  byte = 16*(m&7) + 2*((m>>3)&1) + 256*(m>>4) + 128*((k>>4)&1) + 4*(k>>5) + ((k>>3)&1)
+ *           8-bit operands:   byte = 16*m + (k>>3)
+ *         and the code sits in the low nibble when (k>>2)&1 == 0, else the high nibble.
+ *         sste_meta_to_canonical converts to the plain row-major form
+ *         uint16 [rows, K/16], group g of a row at bits [4(g%4), 4(g%4)+4) of word g/4.
+ */
+#ifndef SSTE_H
+#define SSTE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sste_ctx sste_ctx;
+
+typedef enum {
+    SSTE_OK = 0,
+    SSTE_ERR_INVALID_ARG = 1, /* null pointer, bad enum value */
+    SSTE_ERR_SHAPE = 2,       /* a dimension is not a positive multiple of 128 */
+    SSTE_ERR_DTYPE = 3,       /* dtype combination not supported by this call */
+    SSTE_ERR_ALIGN = 4,       /* pointer not 128-byte aligned */
+    SSTE_ERR_WORKSPACE = 5,   /* workspace missing or too small */
+    SSTE_ERR_ARCH = 6,        /* device is not sm_100 */
+    SSTE_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed */
+    SSTE_ERR_DEGENERATE = 8,  /* beta: S_soft(W) is identically zero; beta was set to 1 */
+    SSTE_ERR_TIMEOUT = 9      /* a bounded device-side wait expired */
+} sste_status;
+
+typedef enum { SSTE_BF16 = 0, SSTE_F32 = 1, SSTE_E4M3 = 2, SSTE_E5M2 = 3 } sste_dtype;
+
+/* Bytes of caller-owned device workspace a context needs (status word + reduction scratch). */
+size_t sste_workspace_bytes(void);
+
+/*
+ * Create a context on `device`.  `workspace` is device memory of at least
+ * sste_workspace_bytes() bytes, 256-byte aligned, owned by the caller and kept
+ * alive until sste_destroy.  The call zeroes the status word (synchronously).
+ * Calls that share a context must be stream-ordered with respect to each other.
+ */
+sste_status sste_create(sste_ctx **ctx, int device, void *workspace, size_t workspace_bytes);
+sste_status sste_destroy(sste_ctx *ctx);
+const char *sste_status_string(sste_status s);
+
+/* Synchronise `stream`, read and clear the device status word.  SSTE_OK if nothing was recorded. */
+sste_status sste_poll_device_status(sste_ctx *ctx, void *stream);
+
+/* Sizes of a compressed operand of a logical [rows, k] matrix. */
+size_t sste_vals_bytes(int rows, int k, sste_dtype dt);
+size_t sste_meta_bytes(int rows, int k);
+
+/*
+ * Eq. 5 (Sec. 4.2, "Minimizing MSE"): beta = <w, S_soft(w)> / ||S_soft(w)||^2 over the whole
+ * tensor, S_soft as in Eq. 4 with groups of four along I.  Products and sums are fp64 in a
+ * fixed order (reproducible run to run); the result is rounded once to fp32 into *beta_dev.
+ * The paper computes beta in the first iteration only and then freezes it (Sec. 4.2,
+ * "Freezing scaling factor"): call this once and keep the scalar.
+ * W: bf16 [O, I].  If S_soft(W) == 0 the call stores 1.0 and records SSTE_ERR_DEGENERATE
+ * in the status word.  Uses the context workspace as scratch.
+ */
+sste_status sste_beta_init(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
+                           float *beta_dev, void *stream);
+
+/*
+ * Eq. 4 + Sec. 4.2: w~ = beta * S_soft(w).  Per group of four along I, t = 2nd-smallest |w|,
+ * s = sign(w) * max(|w| - t, 0) (one fp32 subtraction), w~ = fl32(s * beta)
+ * [FP8: fl32(w~ * wscale)], one round-to-nearest-even cast to `odt` (E4M3: saturating).
+ * Pruned entries are +0.  Kept positions: rank by (|w| descending, index ascending), keep two.
+ * W: bf16 [O, I].  odt: SSTE_BF16 or SSTE_E4M3.  wscale_dev: device float, NULL for bf16.
+ * Outputs: vals [O, I/2] and meta (see top); dense_out (nullable) [O, I] in odt, the operand
+ * of sste_linear_bwd_input.
+ */
+sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
+                                  const float *beta_dev, const float *wscale_dev, sste_dtype odt,
+                                  void *vals, void *meta, void *dense_out, void *stream);
+
+/*
+ * Sec. 5.1: Z = X S(W)^T on sparse tensor cores.  X [T, I], (vals, meta) the compressed w~
+ * [O, I], both of dtype opdt (SSTE_BF16, or SSTE_E4M3 for the FP8 variant).  fp32 accumulation.
+ * Y [T, O] of dtype ydt (SSTE_BF16 or SSTE_F32) = acc * out_scale, out_scale = *out_scale_dev
+ * (NULL means 1; the FP8 variant passes 1/(sx*sw)).
+ */
+sste_status sste_linear_fwd(sste_ctx *ctx, const void *X, int T, const void *vals, const void *meta,
+                            int O, int I, sste_dtype opdt, const float *out_scale_dev,
+                            void *Y, sste_dtype ydt, void *stream);
+
+/*
+ * Sec. 5.1: minimum-variance unbiased 2:4 sparsification of grad_Z^T (the paper applies MVUE to
+ * the output gradient only).  Groups are 4 consecutive tokens of one output column.  Inclusion
+ * probabilities p_i = min(1, c|a_i|), sum 2; kept values a_i / p_i; joint law = systematic
+ * sampling with one uniform per group.  Group (column j, token group tg) has index
+ * g = tg*O + j; Philox4x32-10 with counter (lo32(g>>2), hi32(g>>2), tensor_id, step) and key
+ * (lo32(seed), hi32(seed)); the group uses output word g&3, u = (word >> 8) * 2^-24.
+ * dY: bf16 [T, O].  odt: SSTE_BF16, or SSTE_E5M2 with values fl32(v * gscale) (gscale_dev
+ * non-NULL).  Outputs: the compressed operand of the TRANSPOSED matrix, logical [O, T]:
+ * gvals [O, T/2], gmeta (see top).  dense_q_out (nullable, FP8 only): E5M2(fl32(dY * gscale)) [T, O].
+ */
+sste_status sste_mvue_sparsify(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt,
+                               uint64_t seed, uint32_t tensor_id, uint32_t step,
+                               const float *gscale_dev, sste_dtype odt,
+                               void *gvals, void *gmeta, void *dense_q_out, void *stream);
+
+/*
+ * Sec. 5.1: grad_X = grad_Z S(W), a dense product (the 2:4 structure of S(W) lies along I, which
+ * is not the reduction dimension here).  dY [T, O] of dtype gdt (SSTE_BF16 / SSTE_E5M2),
+ * Wt_dense [O, I] of dtype wdt (SSTE_BF16 / SSTE_E4M3) as written by sste_project_compress.
+ * dX [T, I] of dtype xdt = acc * out_scale.
+ */
+sste_status sste_linear_bwd_input(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt,
+                                  const void *Wt_dense, int I, sste_dtype wdt,
+                                  const float *out_scale_dev, void *dX, sste_dtype xdt, void *stream);
+
+/*
+ * Sec. 5.1: grad_W = MVUE(grad_Z^T) X on sparse tensor cores.  (gvals, gmeta) logical [O, T] of
+ * dtype gdt (SSTE_BF16 / SSTE_E5M2) from sste_mvue_sparsify, X [T, I] of dtype xdt
+ * (SSTE_BF16 / SSTE_E4M3).  dW [O, I] of dtype dwdt (SSTE_BF16 or SSTE_F32) = acc * out_scale.
+ * Straight-through estimator (Eq. 3): this gradient is applied to the dense weight unchanged.
+ */
+sste_status sste_linear_bwd_weight(sste_ctx *ctx, const void *gvals, const void *gmeta, int O, int T,
+                                   sste_dtype gdt, const void *X, int I, sste_dtype xdt,
+                                   const float *out_scale_dev, void *dW, sste_dtype dwdt, void *stream);
+
+/* ---- FP8 whole-process variant (Sec. 5.2): per-tensor rescaling before the cast ---- */
+
+/* *amax_dev = max |x| over n bf16 elements (n % 8 == 0).  Exact, order-free.  amax_dev must hold 0 on entry
+ * or a previous partial maximum to be extended (the call only ever raises it). */
+sste_status sste_amax(sste_ctx *ctx, const void *x, size_t n, sste_dtype dt, float *amax_dev, void *stream);
+
+/* *scale_dev = fl32(fp8_max(odt) / *amax_dev) (1 if amax is 0); *inv_scale_dev (nullable) = fl32(1 / scale). */
+sste_status sste_fp8_scale(sste_ctx *ctx, const float *amax_dev, sste_dtype odt, float *scale_dev,
+                           float *inv_scale_dev, void *stream);
+
+/* q = cast_rn_satfinite(fl32(x * scale)), x bf16, q E4M3 or E5M2; n % 16 == 0. */
+sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n, const float *scale_dev,
+                              sste_dtype odt, void *q, void *stream);
+
+/* *out_dev = fl32(fl32(a * b)) for two device scalars (e.g. the product of two inverse scales). */
+sste_status sste_scalar_mul(sste_ctx *ctx, const float *a_dev, const float *b_dev, float *out_dev, void *stream);
+
+/* ---- test / debug helpers ---- */
+
+/* Operand-image metadata -> canonical uint16 [rows, k/16] (see top).  dt selects the 16-bit or 8-bit image. */
+sste_status sste_meta_to_canonical(sste_ctx *ctx, const void *meta, int rows, int k, sste_dtype dt,
+                                   void *canonical_out, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSTE_H */

@@ -1,0 +1,167 @@
+"""Thin ctypes binding of libsste: same names as the C ABI, argument marshalling only.
+
+Tensors are torch CUDA tensors used purely as device memory (``data_ptr()``);
+every computation runs in the library's kernels on torch's current stream.
+There is no fallback: if the shared library is missing or a call fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_HERE = Path(__file__).resolve().parent
+LIB_PATH = _HERE / "libsste.so"
+
+BF16, F32, E4M3, E5M2 = 0, 1, 2, 3
+OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_DTYPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_DEGENERATE, \
+    ERR_TIMEOUT = range(10)
+
+_TORCH_DT = {BF16: torch.bfloat16, F32: torch.float32, E4M3: torch.float8_e4m3fn, E5M2: torch.float8_e5m2}
+_CODE_OF = {v: k for k, v in _TORCH_DT.items()}
+
+EXPORTS = [
+    "sste_workspace_bytes", "sste_create", "sste_destroy", "sste_status_string", "sste_poll_device_status",
+    "sste_vals_bytes", "sste_meta_bytes", "sste_beta_init", "sste_project_compress", "sste_linear_fwd",
+    "sste_mvue_sparsify", "sste_linear_bwd_input", "sste_linear_bwd_weight", "sste_amax", "sste_fp8_scale",
+    "sste_quantize_fp8", "sste_scalar_mul", "sste_meta_to_canonical",
+]
+
+
+class SsteError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"libsste: {what} (status {code})")
+        self.code = code
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libsste.so from the package directory (built by ``build.py``); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise FileNotFoundError(f"{LIB_PATH} not built: run python -m paper_2409_09099_b200.build")
+        lib = ctypes.CDLL(str(LIB_PATH))
+        lib.sste_workspace_bytes.restype = ctypes.c_size_t
+        lib.sste_vals_bytes.restype = ctypes.c_size_t
+        lib.sste_meta_bytes.restype = ctypes.c_size_t
+        lib.sste_status_string.restype = ctypes.c_char_p
+        _lib = lib
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return ctypes.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous(), "device, contiguous tensors only"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Context:
+    """Owns the device workspace (a torch allocation) and the sste_ctx handle."""
+
+    def __init__(self, device: int = 0):
+        self.lib = load()
+        self.device = device
+        n = self.lib.sste_workspace_bytes()
+        self.workspace = torch.zeros(n, dtype=torch.uint8, device=f"cuda:{device}")
+        handle = ctypes.c_void_p()
+        st = self.lib.sste_create(ctypes.byref(handle), device, _ptr(self.workspace), ctypes.c_size_t(n))
+        self._check(st)
+        self.handle = handle
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.sste_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int):
+        if st != OK:
+            raise SsteError(st, self.lib.sste_status_string(st).decode())
+
+    # ---- hot path -------------------------------------------------------------------------------
+
+    def beta_init(self, W, beta_dev):
+        O, I = W.shape
+        self._check(self.lib.sste_beta_init(self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev), _stream()))
+
+    def project_compress(self, W, beta_dev, vals, meta, dense_out=None, wscale_dev=None):
+        O, I = W.shape
+        self._check(self.lib.sste_project_compress(
+            self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev), _ptr(wscale_dev), _CODE_OF[vals.dtype],
+            _ptr(vals), _ptr(meta), _ptr(dense_out), _stream()))
+
+    def linear_fwd(self, X, vals, meta, Y, out_scale_dev=None):
+        T, I = X.shape
+        O = vals.shape[0]
+        self._check(self.lib.sste_linear_fwd(
+            self.handle, _ptr(X), T, _ptr(vals), _ptr(meta), O, I, _CODE_OF[X.dtype], _ptr(out_scale_dev),
+            _ptr(Y), _CODE_OF[Y.dtype], _stream()))
+
+    def mvue_sparsify(self, dY, seed, tensor_id, step, gvals, gmeta, dense_q_out=None, gscale_dev=None):
+        T, O = dY.shape
+        self._check(self.lib.sste_mvue_sparsify(
+            self.handle, _ptr(dY), T, O, _CODE_OF[dY.dtype], ctypes.c_uint64(seed), ctypes.c_uint32(tensor_id),
+            ctypes.c_uint32(step), _ptr(gscale_dev), _CODE_OF[gvals.dtype], _ptr(gvals), _ptr(gmeta),
+            _ptr(dense_q_out), _stream()))
+
+    def linear_bwd_input(self, dY, Wt_dense, dX, out_scale_dev=None):
+        T, O = dY.shape
+        I = Wt_dense.shape[1]
+        self._check(self.lib.sste_linear_bwd_input(
+            self.handle, _ptr(dY), T, O, _CODE_OF[dY.dtype], _ptr(Wt_dense), I, _CODE_OF[Wt_dense.dtype],
+            _ptr(out_scale_dev), _ptr(dX), _CODE_OF[dX.dtype], _stream()))
+
+    def linear_bwd_weight(self, gvals, gmeta, X, dW, out_scale_dev=None):
+        O = gvals.shape[0]
+        T, I = X.shape
+        self._check(self.lib.sste_linear_bwd_weight(
+            self.handle, _ptr(gvals), _ptr(gmeta), O, T, _CODE_OF[gvals.dtype], _ptr(X), I, _CODE_OF[X.dtype],
+            _ptr(out_scale_dev), _ptr(dW), _CODE_OF[dW.dtype], _stream()))
+
+    # ---- FP8 helpers ----------------------------------------------------------------------------
+
+    def amax(self, x, amax_dev):
+        self._check(self.lib.sste_amax(self.handle, _ptr(x), ctypes.c_size_t(x.numel()), _CODE_OF[x.dtype],
+                                       _ptr(amax_dev), _stream()))
+
+    def fp8_scale(self, amax_dev, odt, scale_dev, inv_scale_dev=None):
+        self._check(self.lib.sste_fp8_scale(self.handle, _ptr(amax_dev), odt, _ptr(scale_dev), _ptr(inv_scale_dev),
+                                            _stream()))
+
+    def quantize_fp8(self, x, scale_dev, q):
+        self._check(self.lib.sste_quantize_fp8(self.handle, _ptr(x), ctypes.c_size_t(x.numel()), _ptr(scale_dev),
+                                               _CODE_OF[q.dtype], _ptr(q), _stream()))
+
+    def scalar_mul(self, a_dev, b_dev, out_dev):
+        self._check(self.lib.sste_scalar_mul(self.handle, _ptr(a_dev), _ptr(b_dev), _ptr(out_dev), _stream()))
+
+    # ---- helpers --------------------------------------------------------------------------------
+
+    def meta_to_canonical(self, meta, rows, k, dt, out):
+        self._check(self.lib.sste_meta_to_canonical(self.handle, _ptr(meta), rows, k, dt, _ptr(out), _stream()))
+
+    def poll_device_status(self) -> int:
+        return self.lib.sste_poll_device_status(self.handle, _stream())
+
+    # ---- allocation helpers (torch as the allocator) ---------------------------------------------
+
+    def alloc_compressed(self, rows, k, dt=BF16):
+        dev = f"cuda:{self.device}"
+        vals = torch.empty((rows, k // 2), dtype=_TORCH_DT[dt], device=dev)
+        meta = torch.empty(self.lib.sste_meta_bytes(rows, k), dtype=torch.uint8, device=dev)
+        return vals, meta

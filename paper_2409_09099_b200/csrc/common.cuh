@@ -1,0 +1,82 @@
+// Shared declarations of libsste's translation units: the context, argument
+// checks and the small device helpers every kernel uses.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp8.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sste.h"
+
+// The context owns nothing but views into the caller's workspace.
+struct sste_ctx {
+    int device;
+    int sm_count;
+    unsigned int *status_dev;   // device status word (first word of the workspace)
+    unsigned int *counter_dev;  // ticket counter of the beta reduction
+    double *partials_dev;       // 2 doubles per reduction block
+    void *cu_tensor_map_encode; // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+constexpr int SSTE_MAX_REDUCE_BLOCKS = 1024;
+constexpr size_t SSTE_WS_STATUS_OFF = 0;
+constexpr size_t SSTE_WS_COUNTER_OFF = 64;
+constexpr size_t SSTE_WS_PARTIALS_OFF = 256;
+constexpr size_t SSTE_WS_BYTES = SSTE_WS_PARTIALS_OFF + 2 * sizeof(double) * SSTE_MAX_REDUCE_BLOCKS;
+
+static inline bool sste_mult128(int v) { return v > 0 && (v % 128) == 0; }
+static inline bool sste_aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+#define SSTE_CUDA_TRY(expr)                         \
+    do {                                            \
+        cudaError_t e__ = (expr);                   \
+        if (e__ != cudaSuccess) return SSTE_ERR_CUDA; \
+    } while (0)
+
+// Make `ctx->device` current for the duration of a call.
+struct sste_device_guard {
+    int prev = -1;
+    bool ok = true;
+    explicit sste_device_guard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        if (prev == dev) prev = -1;
+    }
+    ~sste_device_guard()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+// ---------------------------------------------------------------- device helpers
+
+__device__ __forceinline__ float sste_bf16_bits_to_f32(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+
+// fp32 -> bf16 bits, round to nearest even (finite inputs)
+__device__ __forceinline__ uint32_t sste_f32_to_bf16_bits(float f)
+{
+    return static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(f)));
+}
+
+__device__ __forceinline__ uint32_t sste_f32_to_e4m3(float f)
+{
+    return static_cast<uint32_t>(__nv_cvt_float_to_fp8(f, __NV_SATFINITE, __NV_E4M3));
+}
+
+__device__ __forceinline__ uint32_t sste_f32_to_e5m2(float f)
+{
+    return static_cast<uint32_t>(__nv_cvt_float_to_fp8(f, __NV_SATFINITE, __NV_E5M2));
+}
+
+// Byte offset of (row m, K-offset k) inside a 2 KB metadata atom of 128 rows x 128 logical K.
+__device__ __host__ __forceinline__ uint32_t sste_meta_atom_byte16(uint32_t m, uint32_t k)
+{
+    return 16u * (m & 7u) + 2u * ((m >> 3) & 1u) + 256u * (m >> 4) + 128u * ((k >> 4) & 1u) + 4u * (k >> 5) +
+           ((k >> 3) & 1u);
+}
+__device__ __host__ __forceinline__ uint32_t sste_meta_atom_byte8(uint32_t m, uint32_t k) { return 16u * m + (k >> 3); }
+
+// entry points implemented in the other translation units
+sste_status sste_gemm_launch_check(const sste_ctx *ctx);

@@ -1,0 +1,650 @@
+// HBM-bound kernels of the S-STE linear layer: beta (Eq. 5), the fused
+// projection + scale + 2:4 compression (Eq. 4, Sec. 4.2), the fused MVUE +
+// compression of the output gradient (Sec. 5.1) and the FP8 scaling helpers
+// (Sec. 5.2).  Every fp32 step is a single rounded operation (no FMA
+// contraction) in a fixed order, so results are reproducible bit for bit.
+#include "common.cuh"
+
+namespace {
+
+constexpr int EW_THREADS = 256;
+
+// ---------------------------------------------------------------- group of four: S_soft + kept pair
+
+struct SoftGroup {
+    float w[4];     // beta * S_soft, pruned entries +0
+    uint32_t p0, p1;  // kept positions, p0 < p1
+};
+
+// bits[i]: bf16 bit pattern of a_i (low 16 bits)
+template <bool FP8>
+__device__ __forceinline__ SoftGroup soft_group(const uint32_t bits[4], float beta, float wscale)
+{
+    SoftGroup r;
+    float a[4], m[4];
+    uint32_t key[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        a[i] = sste_bf16_bits_to_f32(bits[i]);
+        m[i] = fabsf(a[i]);
+        key[i] = ((bits[i] & 0x7fffu) << 2) | static_cast<uint32_t>(3 - i);   // magnitude desc, index asc
+    }
+    // second-smallest magnitude without a sort
+    const float lo1 = fminf(m[0], m[1]), hi1 = fmaxf(m[0], m[1]);
+    const float lo2 = fminf(m[2], m[3]), hi2 = fmaxf(m[2], m[3]);
+    const float t = fminf(fmaxf(lo1, lo2), fminf(hi1, hi2));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float d = __fsub_rn(m[i], t);
+        float w = __fmul_rn(copysignf(d, a[i]), beta);
+        if (FP8) w = __fmul_rn(w, wscale);
+        r.w[i] = (d > 0.0f) ? w : 0.0f;
+    }
+    // the two largest keys are kept (keys are pairwise distinct)
+    uint32_t keep = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int above = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) above += (key[j] > key[i]) ? 1 : 0;
+        keep |= (above < 2 ? 1u : 0u) << i;
+    }
+    r.p0 = __ffs(keep) - 1;
+    r.p1 = 31 - __clz(keep);
+    return r;
+}
+
+__device__ __forceinline__ float sel4(uint32_t idx, float v0, float v1, float v2, float v3)
+{
+    return idx == 0 ? v0 : idx == 1 ? v1 : idx == 2 ? v2 : v3;
+}
+
+// ---------------------------------------------------------------- project + compress
+
+// One CTA: 128 rows x 128 input features of W.  Thread = 8 chunks of 8 consecutive features.
+template <bool FP8>
+__global__ void __launch_bounds__(EW_THREADS)
+project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restrict__ beta_dev,
+                        const float *__restrict__ wscale_dev, void *__restrict__ vals, uint8_t *__restrict__ meta,
+                        void *__restrict__ dense)
+{
+    __shared__ __align__(16) uint8_t meta_s[2048];
+    const int tid = threadIdx.x;
+    const int kb = blockIdx.x, rb = blockIdx.y;
+    const float beta = *beta_dev;
+    const float wscale = FP8 ? *wscale_dev : 1.0f;
+    const size_t row_chunks = static_cast<size_t>(I) / 8;
+
+    uint4 in[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int c = i * EW_THREADS + tid;
+        const int row = c >> 4, kc = c & 15;
+        in[i] = __ldg(W + (static_cast<size_t>(rb) * 128 + row) * row_chunks + kb * 16 + kc);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int c = i * EW_THREADS + tid;
+        const int row = c >> 4, kc = c & 15;
+        const uint32_t raw[4] = {in[i].x, in[i].y, in[i].z, in[i].w};
+        uint32_t kept[2][2];   // [group][slot] output bit patterns
+        uint32_t dn[8];        // dense output bit patterns
+        uint32_t mbyte = 0;
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            const uint32_t bits[4] = {raw[2 * g] & 0xffffu, raw[2 * g] >> 16, raw[2 * g + 1] & 0xffffu,
+                                      raw[2 * g + 1] >> 16};
+            const SoftGroup s = soft_group<FP8>(bits, beta, wscale);
+            const float v0 = sel4(s.p0, s.w[0], s.w[1], s.w[2], s.w[3]);
+            const float v1 = sel4(s.p1, s.w[0], s.w[1], s.w[2], s.w[3]);
+            if (FP8) {
+                kept[g][0] = sste_f32_to_e4m3(v0);
+                kept[g][1] = sste_f32_to_e4m3(v1);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) dn[4 * g + e] = sste_f32_to_e4m3(s.w[e]);
+            } else {
+                kept[g][0] = sste_f32_to_bf16_bits(v0);
+                kept[g][1] = sste_f32_to_bf16_bits(v1);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) dn[4 * g + e] = sste_f32_to_bf16_bits(s.w[e]);
+            }
+            mbyte |= (s.p0 | (s.p1 << 2)) << (4 * g);
+        }
+        const uint32_t k = 8u * kc;
+        meta_s[FP8 ? sste_meta_atom_byte8(row, k) : sste_meta_atom_byte16(row, k)] = static_cast<uint8_t>(mbyte);
+        const size_t grow = static_cast<size_t>(rb) * 128 + row;
+        const size_t chunk = grow * row_chunks + kb * 16 + kc;   // index in units of 8 input features
+        if (FP8) {
+            reinterpret_cast<uint32_t *>(vals)[chunk] =
+                kept[0][0] | (kept[0][1] << 8) | (kept[1][0] << 16) | (kept[1][1] << 24);
+            if (dense) {
+                uint2 d;
+                d.x = dn[0] | (dn[1] << 8) | (dn[2] << 16) | (dn[3] << 24);
+                d.y = dn[4] | (dn[5] << 8) | (dn[6] << 16) | (dn[7] << 24);
+                reinterpret_cast<uint2 *>(dense)[chunk] = d;
+            }
+        } else {
+            uint2 v;
+            v.x = kept[0][0] | (kept[0][1] << 16);
+            v.y = kept[1][0] | (kept[1][1] << 16);
+            reinterpret_cast<uint2 *>(vals)[chunk] = v;
+            if (dense) {
+                uint4 d;
+                d.x = dn[0] | (dn[1] << 16);
+                d.y = dn[2] | (dn[3] << 16);
+                d.z = dn[4] | (dn[5] << 16);
+                d.w = dn[6] | (dn[7] << 16);
+                reinterpret_cast<uint4 *>(dense)[chunk] = d;
+            }
+        }
+    }
+    __syncthreads();
+    if (tid < 128) {
+        const size_t atom = static_cast<size_t>(rb) * (I / 128) + kb;
+        reinterpret_cast<uint4 *>(meta + atom * 2048)[tid] = reinterpret_cast<const uint4 *>(meta_s)[tid];
+    }
+}
+
+// ---------------------------------------------------------------- beta
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+
+// fp64 sums of <w, s> and <s, s>, s = S_soft(w) in exact arithmetic; per-block partials are
+// combined by the last block in a fixed order.
+__global__ void __launch_bounds__(EW_THREADS)
+beta_kernel(const uint4 *__restrict__ W, size_t n_chunks, double *__restrict__ partials,
+            unsigned int *__restrict__ counter, float *__restrict__ beta_dev, unsigned int *__restrict__ status)
+{
+    __shared__ double red[2][EW_THREADS / 32];
+    __shared__ bool is_last;
+    double num = 0.0, den = 0.0;
+    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
+         c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const uint4 v = __ldg(W + c);
+        const uint32_t raw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            const uint32_t bits[4] = {raw[2 * g] & 0xffffu, raw[2 * g] >> 16, raw[2 * g + 1] & 0xffffu,
+                                      raw[2 * g + 1] >> 16};
+            double a[4], m[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                a[i] = static_cast<double>(sste_bf16_bits_to_f32(bits[i]));
+                m[i] = fabs(a[i]);
+            }
+            const double lo1 = fmin(m[0], m[1]), hi1 = fmax(m[0], m[1]);
+            const double lo2 = fmin(m[2], m[3]), hi2 = fmax(m[2], m[3]);
+            const double t = fmin(fmax(lo1, lo2), fmin(hi1, hi2));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const double d = m[i] - t;
+                if (d > 0.0) {
+                    const double s = copysign(d, a[i]);
+                    num += a[i] * s;
+                    den += s * s;
+                }
+            }
+        }
+    }
+    num = warp_sum(num);
+    den = warp_sum(den);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { red[0][warp] = num; red[1][warp] = den; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double bn = 0.0, bd = 0.0;
+        for (int w = 0; w < EW_THREADS / 32; ++w) { bn += red[0][w]; bd += red[1][w]; }
+        partials[2 * blockIdx.x] = bn;
+        partials[2 * blockIdx.x + 1] = bd;
+        __threadfence();
+        const unsigned int ticket = atomicAdd(counter, 1u);
+        is_last = (ticket == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (is_last && threadIdx.x < 32) {
+        __threadfence();
+        double tn = 0.0, td = 0.0;
+        for (unsigned int b = threadIdx.x; b < gridDim.x; b += 32) {
+            tn += __ldcg(partials + 2 * b);
+            td += __ldcg(partials + 2 * b + 1);
+        }
+        tn = warp_sum(tn);
+        td = warp_sum(td);
+        if (threadIdx.x == 0) {
+            if (td == 0.0) {
+                *beta_dev = 1.0f;
+                atomicCAS(status, 0u, static_cast<unsigned int>(SSTE_ERR_DEGENERATE));
+            } else {
+                *beta_dev = static_cast<float>(tn / td);
+            }
+            *counter = 0u;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- Philox4x32-10
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                              uint32_t k1, uint32_t out[4])
+{
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        const uint32_t n0 = hi1 ^ c1 ^ k0;
+        const uint32_t n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// ---------------------------------------------------------------- MVUE of one group
+
+struct MvueGroup {
+    uint32_t q0, q1;  // kept positions q0 < q1
+    float v0, v1;     // their values before the cast
+};
+
+__device__ __forceinline__ MvueGroup mvue_group(float a0, float a1, float a2, float a3, float u)
+{
+    const float m0 = fabsf(a0), m1 = fabsf(a1), m2 = fabsf(a2), m3 = fabsf(a3);
+    uint32_t x = 0;
+    float mx = m0;
+    if (m1 > mx) { x = 1; mx = m1; }
+    if (m2 > mx) { x = 2; mx = m2; }
+    if (m3 > mx) { x = 3; mx = m3; }
+    const uint32_t o0 = (x == 0) ? 1u : 0u, o1 = (x <= 1) ? 2u : 1u, o2 = (x <= 2) ? 3u : 2u;
+    const float mo0 = sel4(o0, m0, m1, m2, m3), mo1 = sel4(o1, m0, m1, m2, m3), mo2 = sel4(o2, m0, m1, m2, m3);
+    const float rest = __fadd_rn(__fadd_rn(mo0, mo1), mo2);
+    uint32_t ja, jb;
+    float va, vb;
+    if (mx >= rest) {
+        // clipped: the largest element is kept with probability 1
+        uint32_t second = o0;
+        float val = 0.0f;
+        if (rest != 0.0f) {
+            const float r = __fmul_rn(u, rest);
+            const float c0 = mo0;
+            const float c1 = __fadd_rn(c0, mo1);
+            second = (c0 > r) ? o0 : (c1 > r) ? o1 : o2;
+            float msec = (c0 > r) ? mo0 : (c1 > r) ? mo1 : mo2;
+            if (msec == 0.0f) second = (mo2 > 0.0f) ? o2 : (mo1 > 0.0f) ? o1 : o0;
+            val = copysignf(rest, sel4(second, a0, a1, a2, a3));
+        }
+        ja = x; va = sel4(x, a0, a1, a2, a3);
+        jb = second; vb = val;
+    } else {
+        const float c0 = m0;
+        const float c1 = __fadd_rn(c0, m1);
+        const float c2 = __fadd_rn(c1, m2);
+        const float c3 = __fadd_rn(c2, m3);
+        const float half = __fmul_rn(0.5f, c3);
+        const float r1 = __fmul_rn(u, half);
+        const float r2 = __fadd_rn(r1, half);
+        uint32_t j1 = (c0 > r1) ? 0u : (c1 > r1) ? 1u : (c2 > r1) ? 2u : 3u;
+        uint32_t j2 = 3u;
+        if (j1 < 1u && c1 > r2) j2 = 1u;
+        else if (j1 < 2u && c2 > r2) j2 = 2u;
+        if (j1 == 3u) { j1 = 2u; j2 = 3u; }
+        ja = j1; va = copysignf(half, sel4(j1, a0, a1, a2, a3));
+        jb = j2; vb = copysignf(half, sel4(j2, a0, a1, a2, a3));
+    }
+    MvueGroup r;
+    if (ja < jb) { r.q0 = ja; r.v0 = va; r.q1 = jb; r.v1 = vb; }
+    else         { r.q0 = jb; r.v0 = vb; r.q1 = ja; r.v1 = va; }
+    return r;
+}
+
+// ---------------------------------------------------------------- MVUE + compress (transposing)
+
+// One CTA: 128 tokens x 128 output columns of dY.  A thread task is 4 tokens x 8 columns
+// (8 groups, two Philox calls); results are transposed through shared memory so that every
+// output row (= column of dY) receives whole 128-byte lines.
+template <bool FP8>
+__global__ void __launch_bounds__(EW_THREADS)
+mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t key1, uint32_t tensor_id,
+            uint32_t step, const float *__restrict__ gscale_dev, void *__restrict__ gvals,
+            uint8_t *__restrict__ gmeta, void *__restrict__ dense_q)
+{
+    // bf16: 128 rows x 32 words; fp8: 128 rows x 16 words
+    __shared__ __align__(16) uint32_t vals_s[128 * (FP8 ? 16 : 32)];
+    __shared__ __align__(16) uint8_t meta_s[2048];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int jb = blockIdx.x, tb = blockIdx.y;   // column block, token block
+    const float gscale = FP8 ? *gscale_dev : 1.0f;
+    const size_t row_chunks = static_cast<size_t>(O) / 8;
+
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        const int bidx = it * 8 + warp;
+        const int jc = (bidx & 1) * 8 + (lane & 7);      // column chunk 0..15
+        const int tgl = (bidx >> 1) * 4 + (lane >> 3);   // token group 0..31 inside the tile
+        const size_t tok0 = static_cast<size_t>(tb) * 128 + 4 * tgl;
+        uint4 in[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) in[i] = __ldg(dY + (tok0 + i) * row_chunks + jb * 16 + jc);
+
+        const uint64_t g0 = (static_cast<uint64_t>(tb) * 32 + tgl) * static_cast<uint64_t>(O) +
+                            static_cast<uint64_t>(jb) * 128 + jc * 8;
+        const uint64_t q = g0 >> 2;
+        uint32_t rnd[8];
+        philox4x32_10(static_cast<uint32_t>(q), static_cast<uint32_t>(q >> 32), tensor_id, step, key0, key1, rnd);
+        philox4x32_10(static_cast<uint32_t>(q + 1), static_cast<uint32_t>((q + 1) >> 32), tensor_id, step, key0,
+                      key1, rnd + 4);
+
+        const uint32_t raw[4][4] = {{in[0].x, in[0].y, in[0].z, in[0].w},
+                                    {in[1].x, in[1].y, in[1].z, in[1].w},
+                                    {in[2].x, in[2].y, in[2].z, in[2].w},
+                                    {in[3].x, in[3].y, in[3].z, in[3].w}};
+        uint32_t nibs = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            float a[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t word = raw[i][e >> 1];
+                a[i] = sste_bf16_bits_to_f32((e & 1) ? (word >> 16) : (word & 0xffffu));
+            }
+            const float u = __uint2float_rn(rnd[e] >> 8) * 0x1p-24f;
+            const MvueGroup r = mvue_group(a[0], a[1], a[2], a[3], u);
+            nibs |= (r.q0 | (r.q1 << 2)) << (4 * e);
+            const int jl = jc * 8 + e;
+            if (FP8) {
+                const uint32_t b0 = sste_f32_to_e5m2(__fmul_rn(r.v0, gscale));
+                const uint32_t b1 = sste_f32_to_e5m2(__fmul_rn(r.v1, gscale));
+                reinterpret_cast<uint16_t *>(vals_s)[jl * 32 + (tgl ^ (8 * (jc & 3)))] =
+                    static_cast<uint16_t>(b0 | (b1 << 8));
+            } else {
+                const uint32_t b0 = sste_f32_to_bf16_bits(r.v0);
+                const uint32_t b1 = sste_f32_to_bf16_bits(r.v1);
+                vals_s[jl * 32 + (tgl ^ (4 * (jc & 7)))] = b0 | (b1 << 16);
+            }
+        }
+        if (FP8 && dense_q) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t b[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const uint32_t word = raw[i][e >> 1];
+                    const float v = sste_bf16_bits_to_f32((e & 1) ? (word >> 16) : (word & 0xffffu));
+                    b[e] = sste_f32_to_e5m2(__fmul_rn(v, gscale));
+                }
+                uint2 d;
+                d.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+                d.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
+                reinterpret_cast<uint2 *>(dense_q)[(tok0 + i) * row_chunks + jb * 16 + jc] = d;
+            }
+        }
+        // two token groups share a metadata byte: lane ^ 8 holds the neighbouring token group
+        const uint32_t other = __shfl_xor_sync(0xffffffffu, nibs, 8);
+        if ((tgl & 1) == 0) {
+            const uint32_t k = 4u * tgl;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const uint32_t jl = jc * 8 + e;
+                const uint32_t byte = ((nibs >> (4 * e)) & 0xfu) | (((other >> (4 * e)) & 0xfu) << 4);
+                meta_s[FP8 ? sste_meta_atom_byte8(jl, k) : sste_meta_atom_byte16(jl, k)] = static_cast<uint8_t>(byte);
+            }
+        }
+    }
+    __syncthreads();
+    // rows of the transposed tile: bf16 128 B (8 vectors of 16 B), fp8 64 B (4 vectors)
+    constexpr int VECS = FP8 ? 4 : 8;
+    const size_t out_row_vecs = static_cast<size_t>(T) / (FP8 ? 32 : 16);   // 16-byte vectors per output row
+#pragma unroll
+    for (int it = 0; it < (128 * VECS) / EW_THREADS; ++it) {
+        const int v = it * EW_THREADS + tid;
+        const int row = v / VECS, vec = v % VECS;
+        const int pvec = FP8 ? (vec ^ ((row >> 3) & 3)) : (vec ^ ((row >> 3) & 7));
+        const uint4 data = reinterpret_cast<const uint4 *>(vals_s)[row * VECS + pvec];
+        reinterpret_cast<uint4 *>(gvals)[(static_cast<size_t>(jb) * 128 + row) * out_row_vecs + tb * VECS + vec] = data;
+    }
+    if (tid < 128) {
+        const size_t atom = static_cast<size_t>(jb) * (T / 128) + tb;
+        reinterpret_cast<uint4 *>(gmeta + atom * 2048)[tid] = reinterpret_cast<const uint4 *>(meta_s)[tid];
+    }
+}
+
+// ---------------------------------------------------------------- FP8 helpers
+
+__global__ void __launch_bounds__(EW_THREADS)
+amax_kernel(const uint4 *__restrict__ x, size_t n_chunks, float *__restrict__ amax_dev)
+{
+    uint32_t best = 0;   // magnitude bits of bf16 compare like unsigned integers
+    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
+         c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const uint4 v = __ldg(x + c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            best = max(best, w[i] & 0x7fffu);
+            best = max(best, (w[i] >> 16) & 0x7fffu);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+    if ((threadIdx.x & 31) == 0 && best != 0)
+        atomicMax(reinterpret_cast<unsigned int *>(amax_dev), best << 16);   // non-negative floats order as uints
+}
+
+__global__ void fp8_scale_kernel(const float *amax_dev, float fp8_max, float *scale_dev, float *inv_scale_dev)
+{
+    const float a = *amax_dev;
+    const float s = (a == 0.0f) ? 1.0f : __fdiv_rn(fp8_max, a);
+    *scale_dev = s;
+    if (inv_scale_dev) *inv_scale_dev = __fdiv_rn(1.0f, s);
+}
+
+__global__ void scalar_mul_kernel(const float *a, const float *b, float *out) { *out = __fmul_rn(*a, *b); }
+
+template <bool E5M2>
+__global__ void __launch_bounds__(EW_THREADS)
+quantize_kernel(const uint4 *__restrict__ x, size_t n_chunks, const float *__restrict__ scale_dev,
+                uint2 *__restrict__ q)
+{
+    const float scale = *scale_dev;
+    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
+         c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const uint4 v = __ldg(x + c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t b[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float f = __fmul_rn(sste_bf16_bits_to_f32((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xffffu)), scale);
+            b[i] = E5M2 ? sste_f32_to_e5m2(f) : sste_f32_to_e4m3(f);
+        }
+        uint2 d;
+        d.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+        d.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
+        q[c] = d;
+    }
+}
+
+// ---------------------------------------------------------------- metadata image -> canonical
+
+template <bool EIGHT_BIT>
+__global__ void __launch_bounds__(EW_THREADS)
+meta_to_canonical_kernel(const uint8_t *__restrict__ meta, int rows, int k, uint16_t *__restrict__ out)
+{
+    const size_t words = static_cast<size_t>(rows) * (k / 16);
+    for (size_t w = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; w < words;
+         w += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const uint32_t r = static_cast<uint32_t>(w / (k / 16));
+        const uint32_t kk = static_cast<uint32_t>(w % (k / 16)) * 16;   // first K index of this word
+        const size_t atom = static_cast<size_t>(r >> 7) * (k / 128) + (kk >> 7);
+        const uint8_t *base = meta + atom * 2048;
+        const uint32_t m = r & 127u, ko = kk & 127u;
+        const uint32_t b0 = EIGHT_BIT ? sste_meta_atom_byte8(m, ko) : sste_meta_atom_byte16(m, ko);
+        const uint32_t b1 = EIGHT_BIT ? sste_meta_atom_byte8(m, ko + 8) : sste_meta_atom_byte16(m, ko + 8);
+        out[w] = static_cast<uint16_t>(base[b0] | (base[b1] << 8));
+    }
+}
+
+int grid_for(size_t work_items, int sm_count)
+{
+    size_t blocks = (work_items + EW_THREADS - 1) / EW_THREADS;
+    size_t cap = static_cast<size_t>(sm_count) * 8;
+    if (cap > SSTE_MAX_REDUCE_BLOCKS) cap = SSTE_MAX_REDUCE_BLOCKS;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return static_cast<int>(blocks);
+}
+
+sste_status launch_result() { return cudaGetLastError() == cudaSuccess ? SSTE_OK : SSTE_ERR_CUDA; }
+
+}  // namespace
+
+// ---------------------------------------------------------------- entry points
+
+extern "C" sste_status sste_beta_init(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, float *beta_dev,
+                                      void *stream)
+{
+    if (!ctx || !W || !beta_dev) return SSTE_ERR_INVALID_ARG;
+    if (wdt != SSTE_BF16) return SSTE_ERR_DTYPE;
+    if (!sste_mult128(O) || !sste_mult128(I)) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(W, 128) || !sste_aligned(beta_dev, 4)) return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const size_t n_chunks = static_cast<size_t>(O) * I / 8;
+    const int grid = grid_for(n_chunks, ctx->sm_count);
+    beta_kernel<<<grid, EW_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4 *>(W), n_chunks, ctx->partials_dev, ctx->counter_dev, beta_dev, ctx->status_dev);
+    return launch_result();
+}
+
+extern "C" sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
+                                             const float *beta_dev, const float *wscale_dev, sste_dtype odt,
+                                             void *vals, void *meta, void *dense_out, void *stream)
+{
+    if (!ctx || !W || !beta_dev || !vals || !meta) return SSTE_ERR_INVALID_ARG;
+    if (wdt != SSTE_BF16 || (odt != SSTE_BF16 && odt != SSTE_E4M3)) return SSTE_ERR_DTYPE;
+    if (odt == SSTE_E4M3 && !wscale_dev) return SSTE_ERR_INVALID_ARG;
+    if (!sste_mult128(O) || !sste_mult128(I)) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(W, 128) || !sste_aligned(vals, 128) || !sste_aligned(meta, 128) ||
+        !sste_aligned(dense_out, 128))
+        return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const dim3 grid(I / 128, O / 128);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (odt == SSTE_E4M3)
+        project_compress_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(W), I, beta_dev,
+                                                                   wscale_dev, vals, static_cast<uint8_t *>(meta),
+                                                                   dense_out);
+    else
+        project_compress_kernel<false><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(W), I, beta_dev,
+                                                                    nullptr, vals, static_cast<uint8_t *>(meta),
+                                                                    dense_out);
+    return launch_result();
+}
+
+extern "C" sste_status sste_mvue_sparsify(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt, uint64_t seed,
+                                          uint32_t tensor_id, uint32_t step, const float *gscale_dev, sste_dtype odt,
+                                          void *gvals, void *gmeta, void *dense_q_out, void *stream)
+{
+    if (!ctx || !dY || !gvals || !gmeta) return SSTE_ERR_INVALID_ARG;
+    if (gdt != SSTE_BF16 || (odt != SSTE_BF16 && odt != SSTE_E5M2)) return SSTE_ERR_DTYPE;
+    if (odt == SSTE_E5M2 && !gscale_dev) return SSTE_ERR_INVALID_ARG;
+    if (odt == SSTE_BF16 && dense_q_out) return SSTE_ERR_INVALID_ARG;
+    if (!sste_mult128(O) || !sste_mult128(T)) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(dY, 128) || !sste_aligned(gvals, 128) || !sste_aligned(gmeta, 128) ||
+        !sste_aligned(dense_q_out, 128))
+        return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const dim3 grid(O / 128, T / 128);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint32_t key0 = static_cast<uint32_t>(seed), key1 = static_cast<uint32_t>(seed >> 32);
+    if (odt == SSTE_E5M2)
+        mvue_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(dY), O, T, key0, key1, tensor_id,
+                                                       step, gscale_dev, gvals, static_cast<uint8_t *>(gmeta),
+                                                       dense_q_out);
+    else
+        mvue_kernel<false><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(dY), O, T, key0, key1, tensor_id,
+                                                        step, nullptr, gvals, static_cast<uint8_t *>(gmeta), nullptr);
+    return launch_result();
+}
+
+extern "C" sste_status sste_amax(sste_ctx *ctx, const void *x, size_t n, sste_dtype dt, float *amax_dev, void *stream)
+{
+    if (!ctx || !x || !amax_dev) return SSTE_ERR_INVALID_ARG;
+    if (dt != SSTE_BF16) return SSTE_ERR_DTYPE;
+    if (n == 0 || n % 8 != 0) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(x, 16) || !sste_aligned(amax_dev, 4)) return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const size_t n_chunks = n / 8;
+    amax_kernel<<<grid_for(n_chunks, ctx->sm_count), EW_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4 *>(x), n_chunks, amax_dev);
+    return launch_result();
+}
+
+extern "C" sste_status sste_fp8_scale(sste_ctx *ctx, const float *amax_dev, sste_dtype odt, float *scale_dev,
+                                      float *inv_scale_dev, void *stream)
+{
+    if (!ctx || !amax_dev || !scale_dev) return SSTE_ERR_INVALID_ARG;
+    if (odt != SSTE_E4M3 && odt != SSTE_E5M2) return SSTE_ERR_DTYPE;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    fp8_scale_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(amax_dev, odt == SSTE_E4M3 ? 448.0f : 57344.0f,
+                                                                     scale_dev, inv_scale_dev);
+    return launch_result();
+}
+
+extern "C" sste_status sste_scalar_mul(sste_ctx *ctx, const float *a_dev, const float *b_dev, float *out_dev,
+                                       void *stream)
+{
+    if (!ctx || !a_dev || !b_dev || !out_dev) return SSTE_ERR_INVALID_ARG;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    scalar_mul_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(a_dev, b_dev, out_dev);
+    return launch_result();
+}
+
+extern "C" sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n, const float *scale_dev,
+                                         sste_dtype odt, void *q, void *stream)
+{
+    if (!ctx || !x || !scale_dev || !q) return SSTE_ERR_INVALID_ARG;
+    if (odt != SSTE_E4M3 && odt != SSTE_E5M2) return SSTE_ERR_DTYPE;
+    if (n == 0 || n % 16 != 0) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(x, 16) || !sste_aligned(q, 16)) return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const size_t n_chunks = n / 8;
+    const int grid = grid_for(n_chunks, ctx->sm_count);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (odt == SSTE_E5M2)
+        quantize_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(x), n_chunks, scale_dev,
+                                                           static_cast<uint2 *>(q));
+    else
+        quantize_kernel<false><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(x), n_chunks, scale_dev,
+                                                            static_cast<uint2 *>(q));
+    return launch_result();
+}
+
+extern "C" sste_status sste_meta_to_canonical(sste_ctx *ctx, const void *meta, int rows, int k, sste_dtype dt,
+                                              void *canonical_out, void *stream)
+{
+    if (!ctx || !meta || !canonical_out) return SSTE_ERR_INVALID_ARG;
+    if (!sste_mult128(rows) || !sste_mult128(k)) return SSTE_ERR_SHAPE;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const size_t words = static_cast<size_t>(rows) * (k / 16);
+    const int grid = grid_for(words, ctx->sm_count);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (dt == SSTE_BF16)
+        meta_to_canonical_kernel<false><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint8_t *>(meta), rows, k,
+                                                                     static_cast<uint16_t *>(canonical_out));
+    else
+        meta_to_canonical_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint8_t *>(meta), rows, k,
+                                                                    static_cast<uint16_t *>(canonical_out));
+    return launch_result();
+}
