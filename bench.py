@@ -1,0 +1,364 @@
+#!/usr/bin/env python
+"""Benchmark of the S-STE sparse linear hot path on B200.
+
+One "step" = one pass of the whole path over one batch of the workload:
+for every layer  project+compress -> sparse forward -> MVUE+compress ->
+sparse grad_W -> dense grad_X  (beta is computed once, before timing: the paper
+freezes it after the first iteration).  The default workload is the GPT-2-small
+shaped MLP (two sparse linears, 8 x 1024 tokens, bf16).
+
+Prints ONE JSON line.  `value` is dense-equivalent TFLOP/s (6*T*I*O per layer
+per step) with all inputs resident in HBM; `e2e` is the same metric with the
+inputs starting in pinned host memory and the gradients read back every step.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "S-STE linear fwd+bwd TFLOP/s (dense-equivalent)"
+UNIT = "TFLOP/s"
+KERNELS = ("project_compress", "linear_fwd", "mvue_sparsify", "linear_bwd_weight", "linear_bwd_input")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        super().__init__(daemon=True)
+        self.gpu_index, self.samples, self.reasons, self.proc = gpu_index, [], set(), None
+        self.max_mhz = None
+
+    def run(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+            for line in self.proc.stdout:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    self.samples.append(float(parts[0]))
+                    self.max_mhz = float(parts[1])
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[3:7]):
+                    if val.lower().startswith("active"):
+                        self.reasons.add(name)
+        except FileNotFoundError:
+            pass
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+        self.join(timeout=2)
+        load = sorted(self.samples)
+        return {"sm_mhz": statistics.median(load) if load else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(load)}
+
+
+def workload_layers(cfg_id: int):
+    from paper_2409_09099_b200 import synth
+    return synth.CONFIGS[cfg_id]
+
+
+# --------------------------------------------------------------------------------------------- CPU oracle arm
+
+def oracle_step(tensors, seed, step, fp8=False):
+    """One pass of the path on the CPU oracle for a list of (W, X, dY, beta32) samples."""
+    from oracle import sste_oracle as orc
+    for li, (W, X, dY, beta32) in enumerate(tensors):
+        vals, meta, dense = orc.project_compress(W, beta32)
+        orc.linear_fwd(X, orc.BF16, vals, meta, orc.BF16)
+        gv, gm, _, _ = orc.mvue(dY, seed, li, step)
+        orc.linear_bwd_weight(gv, gm, orc.BF16, X, orc.BF16)
+        orc.linear_bwd_input(dY, orc.BF16, dense, orc.BF16)
+
+
+def oracle_sample(cfg_id: int, tokens: int):
+    import numpy as np
+    from oracle import sste_oracle as orc
+    from paper_2409_09099_b200 import synth
+    cfg = synth.CONFIGS[cfg_id]
+    tensors, flops = [], 0.0
+    for li, L in enumerate(cfg["layers"]):
+        W, X, dY = synth.layer_tensors(cfg_id, li, T=tokens)
+        tensors.append((W, X, dY, np.float32(orc.beta(W)[0])))
+        flops += 6.0 * tokens * L.I * L.O
+    return cfg, tensors, flops
+
+
+def time_oracle(cfg_id: int, tokens: int, steps: int, warmup: int):
+    cfg, tensors, flops = oracle_sample(cfg_id, tokens)
+    for w in range(warmup):
+        oracle_step(tensors, cfg["seed"], w)
+    t0 = time.perf_counter()
+    for s in range(steps):
+        oracle_step(tensors, cfg["seed"], s)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    cores = len(os.sched_getaffinity(0))
+    return dict(value=flops / dt / 1e12, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"config {cfg_id} with {tokens} of {cfg['layers'][0].T} tokens per layer, "
+                       f"{steps} step(s), {dt:.2f} s per step"), dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg_id = args.config
+    cfg = workload_layers(cfg_id)
+    tokens = min(cfg["layers"][0].T, args.ref_tokens)
+    base, dt = time_oracle(cfg_id, tokens, args.steps, min(args.warmup, 1))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg_id, cfg, 1),
+        "cpu_baseline": base,
+        "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg_id, cfg, n_gpus):
+    return {"workload": f"BASELINE config {cfg_id}: " + ", ".join(f"{L.name} W[{L.O},{L.I}] x {L.T} tokens" for L in cfg["layers"]),
+            "precision": "fp8 (e4m3 fwd / e5m2 bwd)" if cfg["fp8"] else "bf16",
+            "tokens_per_gpu": cfg["layers"][0].T, "parallelism": f"dp{n_gpus} (token shards, no data-path collective)",
+            "l2": "flushed between timed steps (512 MiB write)"}
+
+
+# --------------------------------------------------------------------------------------------- GPU arm
+
+def run_gpu(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2409_09099_b200 import binding as B, synth
+    from paper_2409_09099_b200.layer import SsteLinear
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    cfg_id = args.config
+    cfg = synth.CONFIGS[cfg_id]
+    fp8 = cfg["fp8"]
+    ctx = B.Context(local_rank)
+
+    def to_dev(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    # weak scaling: every rank holds the full weights and its own batch of tokens (seeded per rank)
+    layers, host = [], []
+    flops_step = 0.0
+    for li, L in enumerate(cfg["layers"]):
+        W, X, dY = synth.layer_tensors(cfg_id, li)
+        if rank > 0:
+            X = synth.gaussian_bf16(cfg["seed"] * 1000 + 10 * li + 1 + 100 * rank, X.shape, L.sigma_x)
+            dY = synth.gaussian_bf16(cfg["seed"] * 1000 + 10 * li + 2 + 100 * rank, dY.shape, L.sigma_g)
+        lin = SsteLinear(ctx, to_dev(W), L.T, tensor_id=li, seed=cfg["seed"], fp8=fp8)
+        lin.init_beta()
+        layers.append((lin, to_dev(X), to_dev(dY)))
+        host.append(tuple(torch.from_numpy(a.view(np.int16)).pin_memory() for a in (W, X, dY)))
+        flops_step += 6.0 * L.T * L.I * L.O
+    torch.cuda.synchronize()
+
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(step_idx, events=None):
+        """All five calls for every layer; `events` (optional) collects per-kernel CUDA events."""
+        def mark():
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record(stream)
+                events.append(e)
+        for lin, X, dY in layers:
+            mark(); lin.prune()
+            mark(); lin.forward(X)
+            mark()
+            if fp8:
+                lin.backward(dY, step_idx)
+                mark(); mark(); mark()
+            else:
+                c = lin.ctx
+                c.mvue_sparsify(dY, lin.seed, lin.tensor_id, step_idx, lin.gvals, lin.gmeta)
+                mark(); c.linear_bwd_weight(lin.gvals, lin.gmeta, lin.X, lin.dW)
+                mark(); c.linear_bwd_input(dY, lin.w_dense, lin.dX)
+                mark()
+                lin.launches += 3
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for w in range(max(args.warmup, 3)):
+        step(w)
+    barrier()
+    launches_before = sum(l.launches for l, _, _ in layers)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    per_kernel = {k: [] for k in KERNELS}
+    step_ms = []
+    barrier()
+    for s in range(args.steps):
+        flush.zero_()                                   # evict L2 between timed steps
+        ev = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        step(args.warmup + s, ev)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        step_ms.append(e0.elapsed_time(e1))
+        if not fp8:
+            for li in range(len(layers)):
+                base = li * 6
+                for ki, k in enumerate(KERNELS):
+                    per_kernel[k].append((li, ev[base + ki].elapsed_time(ev[base + ki + 1])))
+    barrier()
+    clocks = sampler.stop()
+    gpu_launches = sum(l.launches for l, _, _ in layers) - launches_before
+    total_ms = sum(step_ms)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: inputs start in pinned host memory, gradients are read back ----
+    h2d = sum(sum(t.numel() * 2 for t in h) for h in host)
+    outs = [(torch.empty(l.dW.shape, dtype=torch.int16).pin_memory(), torch.empty(l.dX.shape, dtype=torch.int16).pin_memory())
+            for l, _, _ in layers]
+    d2h = sum(a.numel() * 2 + b.numel() * 2 for a, b in outs)
+
+    def e2e_step(step_idx):
+        for (lin, X, dY), (hW, hX, hdY), (oW, oX) in zip(layers, host, outs):
+            lin.W.view(torch.int16).copy_(hW, non_blocking=True)
+            X.view(torch.int16).copy_(hX, non_blocking=True)
+            dY.view(torch.int16).copy_(hdY, non_blocking=True)
+        step(step_idx)
+        for (lin, _, _), (oW, oX) in zip(layers, outs):
+            oW.copy_(lin.dW.view(torch.int16), non_blocking=True)
+            oX.copy_(lin.dX.view(torch.int16), non_blocking=True)
+
+    e2e_step(0)
+    barrier()
+    e2e_steps = max(2, min(args.steps, 5))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for s in range(e2e_steps):
+        e2e_step(s)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * flops_step / (e2e_ms * 1e-3) / 1e12
+    status = ctx.poll_device_status()
+
+    if rank == 0:
+        peaks = measured_peaks()
+        roofline, breakdown = None, None
+        if not fp8:
+            # share of each kernel in the timed region, and the roofline of the dominant one
+            tot = {k: sum(ms for _, ms in v) for k, v in per_kernel.items()}
+            dom = max(tot, key=tot.get)
+            n_dom = len(per_kernel[dom])
+            avg_ms = tot[dom] / n_dom
+            Ls = cfg["layers"]
+            if dom in ("linear_fwd", "linear_bwd_weight", "linear_bwd_input"):
+                fl = sum(2.0 * L.T * L.I * L.O for L in Ls) / len(Ls)           # dense-equivalent flops per launch (mean)
+                sparse = dom != "linear_bwd_input"
+                peak = peaks["bf16_tflops"] * (2.0 if sparse else 1.0)
+                ach = fl / (avg_ms * 1e-3) / 1e12
+                roofline = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
+                            "frac": ach / peak, "traffic": None,
+                            "peak_source": f"{peaks['source']} cuBLAS bf16 dense burst" + (" x2 (2:4 sparse, nominal ratio)" if sparse else "")}
+            else:
+                per_elt = 5.125 if dom == "project_compress" else 3.125
+                elts = sum((L.O * L.I if dom == "project_compress" else L.T * L.O) for L in Ls) / len(Ls)
+                ach = per_elt * elts / (avg_ms * 1e-3) / 1e9
+                roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                            "peak_source": f"{peaks['source']} copy bandwidth"}
+            breakdown = {k: {"ms_per_step": tot[k] / args.steps, "share": tot[k] / sum(tot.values())} for k in KERNELS}
+        cpu_base = None
+        if world == 1 or rank == 0:
+            cpu_base, _ = time_oracle(cfg_id, min(cfg["layers"][0].T, args.ref_tokens), 5, 1)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "fp8" if fp8 else "bf16", "data": "synthetic",
+            "config": workload_config(cfg_id, cfg, world),
+            "pct_of_sparse_peak_nominal": 100.0 * value / world / 4500.0,
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms},
+            "gpu_launches": gpu_launches,
+            "roofline": roofline,
+            "kernels": breakdown,
+            "cpu_baseline": cpu_base,
+            "device_status": status,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="BASELINE config id (2 = GPT-2-small MLP, the default workload)")
+    ap.add_argument("--ref-tokens", type=int, default=8192, help="tokens per layer in the CPU-oracle sample")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

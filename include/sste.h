@@ -161,8 +161,8 @@ sste_status sste_linear_bwd_weight(sste_ctx *ctx, const void *gvals, const void 
 
 /* ---- FP8 whole-process variant (Sec. 5.2): per-tensor rescaling before the cast ---- */
 
-/* *amax_dev = max |x| over n bf16 elements (n % 8 == 0).  Exact, order-free.  amax_dev must hold 0 on entry
- * or a previous partial maximum to be extended (the call only ever raises it). */
+/* *amax_dev = max |x| over n bf16 elements (n % 8 == 0).  Exact, order-free.  The call first sets
+ * *amax_dev to 0 on the stream, then raises it with an atomic maximum. */
 sste_status sste_amax(sste_ctx *ctx, const void *x, size_t n, sste_dtype dt, float *amax_dev, void *stream);
 
 /* *scale_dev = fl32(fp8_max(odt) / *amax_dev) (1 if amax is 0); *inv_scale_dev (nullable) = fl32(1 / scale). */

@@ -582,6 +582,7 @@ extern "C" sste_status sste_amax(sste_ctx *ctx, const void *x, size_t n, sste_dt
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
     const size_t n_chunks = n / 8;
+    SSTE_CUDA_TRY(cudaMemsetAsync(amax_dev, 0, sizeof(float), static_cast<cudaStream_t>(stream)));
     amax_kernel<<<grid_for(n_chunks, ctx->sm_count), EW_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4 *>(x), n_chunks, amax_dev);
     return launch_result();

@@ -1,0 +1,108 @@
+"""One S-STE linear layer as a user of the library sees it: buffers + the call sequence.
+
+This is bookkeeping only (which buffer goes to which C-ABI call, in the order the
+paper's training iteration prescribes); every computation runs in libsste.
+Straight-through estimator (Eq. 3): ``dW`` is the gradient with respect to the
+sparse weight and is meant to be applied to the dense weight unchanged.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class SsteLinear:
+    """W[O, I] dense master weight (bf16); forward Y = X S(W)^T, backward (dX, dW).
+
+    ``fp8=True`` selects the whole-process FP8 variant (Sec. 5.2): E4M3 forward
+    operands, E5M2 output gradient, per-tensor scale = fp8_max / amax computed
+    just in time on the device.
+    """
+
+    def __init__(self, ctx: B.Context, W: torch.Tensor, T: int, tensor_id: int = 0, seed: int = 0,
+                 fp8: bool = False, out_dtype: torch.dtype = torch.bfloat16):
+        assert W.dtype == torch.bfloat16 and W.is_cuda
+        self.ctx, self.W, self.T, self.tensor_id, self.seed, self.fp8 = ctx, W, T, tensor_id, seed, fp8
+        self.O, self.I = W.shape
+        O, I, dev = self.O, self.I, W.device
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.beta = torch.zeros(1, **f32)
+        self.beta_ready = False
+        wdt = B.E4M3 if fp8 else B.BF16
+        gdt = B.E5M2 if fp8 else B.BF16
+        self.vals, self.meta = ctx.alloc_compressed(O, I, wdt)
+        self.w_dense = torch.empty((O, I), dtype=B._TORCH_DT[wdt], device=dev)
+        self.gvals, self.gmeta = ctx.alloc_compressed(O, T, gdt)
+        self.Y = torch.empty((T, O), dtype=out_dtype, device=dev)
+        self.dX = torch.empty((T, I), dtype=out_dtype, device=dev)
+        self.dW = torch.empty((O, I), dtype=out_dtype, device=dev)
+        self.launches = 0
+        if fp8:
+            self.amax = torch.zeros(3, **f32)          # X, w~ (through W and beta), dY
+            self.scale = torch.ones(3, **f32)
+            self.inv = torch.ones(3, **f32)
+            self.inv_xw = torch.ones(1, **f32)
+            self.inv_gx = torch.ones(1, **f32)
+            self.inv_gw = torch.ones(1, **f32)
+            self.Xq = torch.empty((T, I), dtype=torch.float8_e4m3fn, device=dev)
+            self.dYq = torch.empty((T, O), dtype=torch.float8_e5m2, device=dev)
+            self.w_tilde = torch.empty((O, I), dtype=torch.bfloat16, device=dev)
+            self._v16, self._m16 = ctx.alloc_compressed(O, I, B.BF16)
+
+    # (0) first iteration only: beta is computed once and then frozen (Sec. 4.2)
+    def init_beta(self):
+        self.ctx.beta_init(self.W, self.beta)
+        self.beta_ready = True
+        self.launches += 1
+
+    # (1) prune: w~ = beta * S_soft(W), compressed for the sparse products, dense for grad_X
+    def prune(self):
+        assert self.beta_ready, "call init_beta() in the first iteration"
+        c = self.ctx
+        if not self.fp8:
+            c.project_compress(self.W, self.beta, self.vals, self.meta, self.w_dense)
+            self.launches += 1
+            return
+        # FP8: the scale of w~ needs amax(w~): project once to bf16, take amax, project again to E4M3
+        c.project_compress(self.W, self.beta, self._v16, self._m16, self.w_tilde)
+        c.amax(self.w_tilde, self.amax[1:2])
+        c.fp8_scale(self.amax[1:2], B.E4M3, self.scale[1:2], self.inv[1:2])
+        c.project_compress(self.W, self.beta, self.vals, self.meta, self.w_dense, wscale_dev=self.scale[1:2])
+        self.launches += 4
+
+    # (2a) forward with the sparse weight
+    def forward(self, X):
+        c = self.ctx
+        if not self.fp8:
+            self.X = X
+            c.linear_fwd(X, self.vals, self.meta, self.Y)
+            self.launches += 1
+            return self.Y
+        c.amax(X, self.amax[0:1])
+        c.fp8_scale(self.amax[0:1], B.E4M3, self.scale[0:1], self.inv[0:1])
+        c.quantize_fp8(X, self.scale[0:1], self.Xq)
+        c.scalar_mul(self.inv[0:1], self.inv[1:2], self.inv_xw)
+        c.linear_fwd(self.Xq, self.vals, self.meta, self.Y, out_scale_dev=self.inv_xw)
+        self.launches += 5
+        return self.Y
+
+    # (2b) backward: MVUE on the output gradient for grad_W, dense product for grad_X
+    def backward(self, dY, step: int = 0):
+        c = self.ctx
+        if not self.fp8:
+            c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta)
+            c.linear_bwd_weight(self.gvals, self.gmeta, self.X, self.dW)
+            c.linear_bwd_input(dY, self.w_dense, self.dX)
+            self.launches += 3
+            return self.dX, self.dW
+        c.amax(dY, self.amax[2:3])
+        c.fp8_scale(self.amax[2:3], B.E5M2, self.scale[2:3], self.inv[2:3])
+        c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta, dense_q_out=self.dYq,
+                        gscale_dev=self.scale[2:3])
+        c.scalar_mul(self.inv[2:3], self.inv[0:1], self.inv_gx)
+        c.scalar_mul(self.inv[2:3], self.inv[1:2], self.inv_gw)
+        c.linear_bwd_weight(self.gvals, self.gmeta, self.Xq, self.dW, out_scale_dev=self.inv_gx)
+        c.linear_bwd_input(self.dYq, self.w_dense, self.dX, out_scale_dev=self.inv_gw)
+        self.launches += 7
+        return self.dX, self.dW

@@ -1,0 +1,185 @@
+"""GPU parity: every libsste call, through the C ABI, against the CPU oracle on the same seeded inputs.
+
+Bar: bit-exact for projected values, metadata, MVUE outputs and FP8 codes (given the same fp32
+beta / scales); beta within 1e-6 relative; products within a relative Frobenius error of 1e-2
+(bf16) / 5e-2 (FP8) of the fp64 product of the same operand bits.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sste_oracle as orc
+from paper_2409_09099_b200 import synth
+from tests.gpu_util import DEV, bits16, bits8, canonical_meta, dbf16, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+BF16_GEMM_TOL = 1e-2      # relative Frobenius error vs the fp64 product, bf16 operands and bf16 output
+FP8_GEMM_TOL = 5e-2
+BETA_TOL = 1e-6
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2409_09099_b200 import binding
+    c = binding.Context(0)
+    yield c
+    assert c.poll_device_status() == 0
+    c.close()
+
+
+def _adversarial_weight(seed, O, I):
+    """Gaussian weights with exact ties, zeros, an all-equal row and an all-zero row."""
+    W = synth.bf16_bits_to_f32(synth.gaussian_bf16(seed, (O, I), 0.02))
+    rng = np.random.default_rng(seed + 99)
+    mask = rng.random(W.shape) < 0.15
+    W[mask] = np.round(W[mask] * 128) / 128          # coarse grid: many ties inside groups
+    W[::7, ::3] = 0.0
+    W[3] = 0.25
+    W[5] = 0.0
+    W[6, ::2] = -0.0
+    return synth.to_bf16_bits(W)
+
+
+SHAPES = [(256, 256, 512), (384, 640, 1152), (128, 128, 128)]   # (O, I, T): config 1, a ragged multi-tile case, one tile
+
+
+@pytest.mark.parametrize("O,I,T", SHAPES)
+def test_beta_and_project_compress(ctx, O, I, T):
+    from paper_2409_09099_b200 import binding as B
+    W = _adversarial_weight(O + I, O, I)
+    Wd = dbf16(W)
+    beta_dev = torch.zeros(1, dtype=torch.float32, device=DEV)
+    ctx.beta_init(Wd, beta_dev)
+    b_ref = orc.beta(W)[0]
+    assert abs(beta_dev.item() - b_ref) <= BETA_TOL * abs(b_ref)
+    # reproducible run to run (fixed reduction order)
+    beta2 = torch.zeros(1, dtype=torch.float32, device=DEV)
+    ctx.beta_init(Wd, beta2)
+    assert beta2.item() == beta_dev.item()
+    beta32 = np.float32(beta_dev.item())
+    vals, meta = ctx.alloc_compressed(O, I)
+    dense = torch.empty((O, I), dtype=torch.bfloat16, device=DEV)
+    ctx.project_compress(Wd, beta_dev, vals, meta, dense)
+    ov, om, od = orc.project_compress(W, beta32)
+    assert np.array_equal(bits16(vals), ov)
+    assert np.array_equal(canonical_meta(ctx, meta, O, I, B.BF16), om)
+    assert np.array_equal(bits16(dense), od)
+    # dense_out is optional
+    vals2, meta2 = ctx.alloc_compressed(O, I)
+    ctx.project_compress(Wd, beta_dev, vals2, meta2, None)
+    assert torch.equal(vals2.view(torch.int16), vals.view(torch.int16)) and torch.equal(meta2, meta)
+
+
+def test_beta_degenerate_and_sparse_input(ctx):
+    O = I = 128
+    beta_dev = torch.zeros(1, dtype=torch.float32, device=DEV)
+    ctx.beta_init(dbf16(synth.to_bf16_bits(np.full((O, I), 2.0, np.float32))), beta_dev)
+    assert beta_dev.item() == 1.0
+    assert ctx.poll_device_status() == 8          # SSTE_ERR_DEGENERATE recorded, then cleared
+    assert ctx.poll_device_status() == 0
+    W = synth.bf16_bits_to_f32(synth.gaussian_bf16(4, (O, I), 0.02)).reshape(O, I // 4, 4)
+    W[:, :, [1, 2]] = 0
+    ctx.beta_init(dbf16(synth.to_bf16_bits(W.reshape(O, I))), beta_dev)
+    assert beta_dev.item() == 1.0 and ctx.poll_device_status() == 0
+
+
+@pytest.mark.parametrize("O,I,T", SHAPES)
+def test_mvue_sparsify(ctx, O, I, T):
+    from paper_2409_09099_b200 import binding as B
+    dY = synth.bf16_bits_to_f32(synth.gaussian_bf16(T + O, (T, O), 1e-2))
+    dY[::5, ::3] = 0.0                      # groups with zeros
+    dY[8:12, 7] = 0.0                       # an all-zero group
+    dY[12:16, 9] = [0.0, 3.0, 0.0, 0.0]     # one nonzero
+    dY[16:20, 11] = 0.5                     # all equal
+    dY[20:24, 13] = [4.0, -0.5, 0.25, 1.0]  # clipped
+    dY = synth.to_bf16_bits(dY)
+    seed, tid, step = (0xABCD << 32) | 0x1234, 5, 17
+    gvals, gmeta = ctx.alloc_compressed(O, T)
+    ctx.mvue_sparsify(dbf16(dY), seed, tid, step, gvals, gmeta)
+    ogv, ogm, _, _ = orc.mvue(dY, seed, tid, step)
+    assert np.array_equal(bits16(gvals), ogv)
+    assert np.array_equal(canonical_meta(ctx, gmeta, O, T, B.BF16), ogm)
+    # another step draws other bits
+    gvals2, gmeta2 = ctx.alloc_compressed(O, T)
+    ctx.mvue_sparsify(dbf16(dY), seed, tid, step + 1, gvals2, gmeta2)
+    assert not torch.equal(gmeta2, gmeta)
+    assert np.array_equal(bits16(gvals2), orc.mvue(dY, seed, tid, step + 1)[0])
+
+
+@pytest.mark.parametrize("O,I,T", SHAPES)
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_three_products(ctx, O, I, T, out_dtype):
+    from paper_2409_09099_b200 import binding as B
+    W, X, dY = _adversarial_weight(O, O, I), synth.gaussian_bf16(O + 1, (T, I), 1.0), synth.gaussian_bf16(O + 2, (T, O), 1e-2)
+    Wd, Xd, dYd = dbf16(W), dbf16(X), dbf16(dY)
+    beta_dev = torch.zeros(1, dtype=torch.float32, device=DEV)
+    ctx.beta_init(Wd, beta_dev)
+    vals, meta = ctx.alloc_compressed(O, I)
+    dense = torch.empty((O, I), dtype=torch.bfloat16, device=DEV)
+    ctx.project_compress(Wd, beta_dev, vals, meta, dense)
+    gvals, gmeta = ctx.alloc_compressed(O, T)
+    ctx.mvue_sparsify(dYd, 7, 1, 0, gvals, gmeta)
+    Y = torch.empty((T, O), dtype=out_dtype, device=DEV)
+    dW = torch.empty((O, I), dtype=out_dtype, device=DEV)
+    dX = torch.empty((T, I), dtype=out_dtype, device=DEV)
+    ctx.linear_fwd(Xd, vals, meta, Y)
+    ctx.linear_bwd_weight(gvals, gmeta, Xd, dW)
+    ctx.linear_bwd_input(dYd, dense, dX)
+    torch.cuda.synchronize()
+    # the oracle multiplies the SAME operand bits (already verified bit-exact above) in fp64
+    Y_ref = orc.linear_fwd(X, orc.BF16, bits16(vals), canonical_meta(ctx, meta, O, I, B.BF16), orc.BF16)
+    dW_ref = orc.linear_bwd_weight(bits16(gvals), canonical_meta(ctx, gmeta, O, T, B.BF16), orc.BF16, X, orc.BF16)
+    dX_ref = orc.linear_bwd_input(dY, orc.BF16, bits16(dense), orc.BF16)
+    tol = BF16_GEMM_TOL if out_dtype == torch.bfloat16 else 1e-5
+    assert rel_fro(Y.float().cpu().numpy(), Y_ref) <= tol
+    assert rel_fro(dW.float().cpu().numpy(), dW_ref) <= tol
+    assert rel_fro(dX.float().cpu().numpy(), dX_ref) <= tol
+    # element-wise too: no entry is off by more than bf16 rounding of the accumulated value
+    for got, ref in ((Y, Y_ref), (dW, dW_ref), (dX, dX_ref)):
+        g = got.float().cpu().numpy().astype(np.float64)
+        bound = 2.0 ** -7 * np.abs(ref) + 1e-4 * np.abs(ref).max()
+        assert (np.abs(g - ref) <= bound).all()
+    # output scale factor
+    sc = torch.tensor([0.25], dtype=torch.float32, device=DEV)
+    Y2 = torch.empty_like(Y)
+    ctx.linear_fwd(Xd, vals, meta, Y2, out_scale_dev=sc)
+    assert torch.equal(Y2.float(), Y.float() * 0.25)
+
+
+def test_forward_of_already_sparse_weight_is_the_dense_product(ctx):
+    """W already 2:4 => beta = 1, S(W) = W: the sparse forward equals the plain product X W^T."""
+    O, I, T = 256, 512, 384
+    W = synth.bf16_bits_to_f32(synth.gaussian_bf16(41, (O, I), 0.02)).reshape(O, I // 4, 4)
+    W[:, :, [0, 3]] = 0
+    W = synth.to_bf16_bits(W.reshape(O, I))
+    X = synth.gaussian_bf16(42, (T, I), 1.0)
+    beta_dev = torch.zeros(1, dtype=torch.float32, device=DEV)
+    ctx.beta_init(dbf16(W), beta_dev)
+    assert beta_dev.item() == 1.0
+    vals, meta = ctx.alloc_compressed(O, I)
+    ctx.project_compress(dbf16(W), beta_dev, vals, meta, None)
+    Y = torch.empty((T, O), dtype=torch.float32, device=DEV)
+    ctx.linear_fwd(dbf16(X), vals, meta, Y)
+    ref = synth.bf16_bits_to_f32(X).astype(np.float64) @ synth.bf16_bits_to_f32(W).astype(np.float64).T
+    assert rel_fro(Y.cpu().numpy(), ref) <= 1e-5
+
+
+def test_argument_validation_launches_nothing(ctx):
+    from paper_2409_09099_b200 import binding as B
+    W = torch.zeros((128, 128), dtype=torch.bfloat16, device=DEV)
+    beta = torch.ones(1, dtype=torch.float32, device=DEV)
+    vals, meta = ctx.alloc_compressed(128, 128)
+    with pytest.raises(B.SsteError) as e:
+        ctx.project_compress(torch.zeros((128, 192), dtype=torch.bfloat16, device=DEV), beta, vals, meta)
+    assert e.value.code == B.ERR_SHAPE
+    with pytest.raises(B.SsteError) as e:      # misaligned output pointer
+        ctx.project_compress(W, beta, vals.view(-1)[4:4 + 128 * 32].view(128, 32), meta)
+    assert e.value.code in (B.ERR_ALIGN, B.ERR_SHAPE)
+    with pytest.raises(B.SsteError) as e:      # E5M2 is not a forward operand type
+        ctx.linear_fwd(torch.zeros((128, 128), dtype=torch.float8_e5m2, device=DEV),
+                       torch.zeros((128, 64), dtype=torch.float8_e5m2, device=DEV), meta,
+                       torch.zeros((128, 128), dtype=torch.bfloat16, device=DEV))
+    assert e.value.code == B.ERR_DTYPE
+    assert ctx.lib.sste_beta_init(ctx.handle, None, 128, 128, 0, None, None) == B.ERR_INVALID_ARG
+    assert ctx.poll_device_status() == 0
