@@ -2,10 +2,17 @@
 //   forward      Z^T = S(W) X^T              sparse A (values + metadata), K-major B
 //   grad weight  grad_W = MVUE(grad_Z^T) X   sparse A, MN-major B
 //   grad input   grad_X = grad_Z S(W)        dense A, MN-major B
-// One persistent, warp-specialised kernel template: a TMA producer warp fills a
-// shared-memory ring, one thread issues tcgen05.mma / tcgen05.mma.sp with fp32
-// accumulators in tensor memory, four warps drain the accumulators.  The 2:4
-// metadata travels HBM -> shared memory (bulk copy) -> tensor memory (tcgen05.cp).
+//
+// One persistent, warp-specialised kernel template run by CTA PAIRS (cluster of two,
+// tcgen05 cta_group::2).  A pair owns a 256 x 256 output tile: each CTA holds its own
+// 128 rows of A and HALF of the B tile, so the B operand is streamed from shared memory
+// at half the rate per SM -- with one CTA per tile the sparse instruction is bound by that
+// stream and runs no faster than the dense one -- and L2 -> SM traffic per flop drops.
+//   warp 0    TMA producer (both CTAs; all transaction bytes land on the leader's barrier)
+//   warp 1    leader CTA: tcgen05.mma[.sp] issue; both CTAs: tensor-memory allocation
+//   warps 2-5 epilogue: TMEM -> registers -> bf16 -> shared memory -> TMA store
+//   warps 6-9 (sparse only) metadata: HBM -> registers -> tensor memory (tcgen05.st), so that no
+//             metadata copy sits between two MMAs in the tensor pipe (a tcgen05.cp there drains it)
 // Every wait is bounded: on expiry the CTA records SSTE_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 
@@ -13,9 +20,12 @@
 
 namespace {
 
-constexpr int BM = 128;            // rows of A per tile (= UMMA M)
-constexpr int GEMM_THREADS = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr int BM = 128;            // rows of A per CTA (a pair covers 256)
+constexpr int BN = 256;            // columns per tile (each CTA stages BN/2 of B)
 constexpr int TMEM_COLS = 512;
+constexpr int META_COL0 = 256;     // accumulators occupy tensor-memory columns [0, 256)
+constexpr int META_REGIONS = 8;   // metadata regions of 16 columns (four atoms) after the accumulators
+constexpr int STAGING_BYTES = 32768;   // half of one CTA's bf16 output tile: 128 x 128 x 2
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
 
 enum class BMajor { K, MN };
@@ -23,6 +33,24 @@ enum class BMajor { K, MN };
 // ------------------------------------------------------------------ PTX wrappers
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
@@ -32,23 +60,27 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+// arrive on a barrier that may live in the peer CTA (shared::cluster address)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// One try: the thread is suspended by the hardware until the phase completes or a time limit of
+// about a millisecond passes, so a waiting thread does not poll shared memory (the sparse MMA streams
+// its operands at 3/4 of the shared-memory bandwidth and is slowed down by pollers).
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(1000000u)
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false (after recording a timeout) instead of spinning forever.
+// Bounded wait of ONE thread.  Returns false (after recording a timeout) instead of spinning forever.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned int *status, volatile int *abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;
@@ -63,60 +95,75 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigne
         }
     }
 }
+// Bounded wait of a whole warp: lane 0 waits, the others park at the warp barrier.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, unsigned int *status, volatile int *abort_flag)
+{
+    uint32_t ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, status, abort_flag) ? 1u : 0u;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
+}
 
+// 2-D tiled TMA load into this CTA's shared memory; the transaction bytes are signalled on
+// `bar`, which may be the pair leader's barrier (cta_group::2 form).
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
 {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y)
                  : "memory");
 }
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
+__device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
 {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tmem_relinquish()
 {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
 {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// arrive on an mbarrier once all tcgen05 operations issued so far by this thread have completed
-__device__ __forceinline__ void tc_commit(uint32_t bar)
+// Arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once every
+// tcgen05 operation issued so far by this thread has completed.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// shared memory -> tensor memory, 128 lanes x 16 bytes
-__device__ __forceinline__ void tc_cp_128x128b(uint32_t taddr, uint64_t sdesc)
-{
-    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(static_cast<uint16_t>(3))
+        : "memory");
 }
 template <bool F8>
 __device__ __forceinline__ void tc_mma_dense(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate)
 {
     if (F8)
         asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+                     "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
                      ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
     else
         asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                      ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
 }
 template <bool F8>
@@ -125,11 +172,11 @@ __device__ __forceinline__ void tc_mma_sparse(uint32_t d, uint64_t a, uint64_t b
 {
     if (F8)
         asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                     "tcgen05.mma.sp.cta_group::1.kind::f8f6f4 [%0], %1, %2, [%3], %4, p;\n\t}"
+                     "tcgen05.mma.sp.cta_group::2.kind::f8f6f4 [%0], %1, %2, [%3], %4, p;\n\t}"
                      ::"r"(d), "l"(a), "l"(b), "r"(e), "r"(idesc), "r"(accumulate) : "memory");
     else
         asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                     "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+                     "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
                      ::"r"(d), "l"(a), "l"(b), "r"(e), "r"(idesc), "r"(accumulate) : "memory");
 }
 // 32 lanes x 32 consecutive 32-bit columns -> 32 registers per thread
@@ -159,74 +206,112 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 
 // Instruction descriptor: sparse selector [0,2), sparse flag [2], D = fp32 [4,6), A format [7,10),
 // B format [10,13), A major [15], B major [16] (1 = MN-major), N>>3 [17,23), M>>4 [24,29).
-__host__ __device__ constexpr uint32_t instr_desc(bool sparse, uint32_t afmt, uint32_t bfmt, bool b_mn_major, int n)
+// M is 256: the pair's two 128-row halves.
+__host__ __device__ constexpr uint32_t instr_desc(bool sparse, uint32_t afmt, uint32_t bfmt, bool b_mn_major)
 {
     return (sparse ? 4u : 0u) | (1u << 4) | (afmt << 7) | (bfmt << 10) | ((b_mn_major ? 1u : 0u) << 16) |
-           (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
+           (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>((2 * BM) >> 4) << 24);
 }
 
 // ------------------------------------------------------------------ kernel
 
 struct GemmParams {
     int M, N, K;            // logical problem: D[M, N] = A[M, K] * B
-    const uint8_t *meta;    // metadata image of A (sparse only)
-    void *D;                // output
+    void *D;                // output (used by the direct-store fp32 epilogue)
     const float *out_scale; // device scalar or null
     unsigned int *status;
     uint32_t afmt, bfmt;    // operand format codes of the instruction descriptor
+#ifdef SSTE_PROBE
+    int probe;              // 1: skip the loads after the first ring fill, 2: skip the MMAs
+    long long *dbg;         // clock64 stamps of pair 0: [tile][0..3] = mma start, mma issued, acc full seen, epilogue done
+#endif
 };
+#ifdef SSTE_PROBE
+int g_probe_mode = 0;
+long long *g_probe_dbg = nullptr;
+#define PROBE_MODE(p) ((p).probe)
+#define PROBE_STAMP(p, tile, k) do { if ((p).dbg && blockIdx.x == 0 && (tile) < 16) (p).dbg[(tile) * 4 + (k)] = clock64(); } while (0)
+#else
+#define PROBE_MODE(p) 0
+#define PROBE_STAMP(p, tile, k) do { } while (0)
+#endif
 
-template <bool SPARSE, int BN>
+// 32 lanes x 4 consecutive 32-bit columns <- 4 registers per thread
+__device__ __forceinline__ void tmem_st_32x4(uint32_t taddr, uint4 v)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
+                 ::"r"(taddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory plan of one CTA.  A stage holds 128 bytes of K per A row and, for the sparse
+// kernels, two B sub-tiles of 128 bytes of K each (the compressed A row covers twice the K of
+// one B row); the dense kernel pairs it with one B sub-tile.
+template <bool SPARSE>
 struct Cfg {
-    static constexpr int A_STAGE = SPARSE ? 8192 : 16384;       // 128 rows x (64 | 128) bytes
-    static constexpr int B_STAGE = BN * 128;                    // BN rows x 128 bytes (or 128 B x BK rows per chunk)
-    static constexpr int META_STAGE = SPARSE ? 2048 : 0;
-    static constexpr int STAGE = A_STAGE + B_STAGE + META_STAGE;
-    static constexpr int STAGES = (BN == 256) ? (SPARSE ? 5 : 4) : (SPARSE ? 8 : 6);
-    static constexpr int ACC_BUFS = (BN == 256) ? 1 : 2;
-    static constexpr int META_COL0 = 256;                       // accumulators occupy columns [0, 256)
-    static constexpr int SMEM_BYTES = STAGES * STAGE + 1024 /* alignment slack */ + 256 /* barriers */;
+    static constexpr int A_STAGE = 16384;                        // 128 rows x 128 bytes
+    static constexpr int B_SUB = (BN / 2) * 128;                 // this CTA's half of one B sub-tile
+    static constexpr int B_STAGE = SPARSE ? 2 * B_SUB : B_SUB;
+    static constexpr int STAGE = A_STAGE + B_STAGE;
+    static constexpr int STAGES = SPARSE ? 4 : 6;
+    static constexpr int THREADS = SPARSE ? 320 : 192;           // + 4 metadata warps for the sparse kernels
+    static constexpr int SMEM_BYTES = STAGES * STAGE + STAGING_BYTES + 1024 /* alignment slack */ + 512 /* barriers */;
 };
 
 // ELT: operand element size in bytes (2 = bf16 via kind::f16, 1 = fp8 via kind::f8f6f4).
-// OUT_T: store D transposed (out[n, m]); OUT_F32: fp32 output instead of bf16.
-template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+// OUT_T: store D transposed (out[n, m]); OUT_F32: fp32 output (direct stores) instead of bf16 (TMA stores).
+template <bool SPARSE, BMajor BMAJ, int ELT, bool OUT_T, bool OUT_F32>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Cfg<SPARSE>::THREADS, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const __grid_constant__ CUtensorMap map_d, const uint8_t *__restrict__ meta, const GemmParams p)
 {
-    using C = Cfg<SPARSE, BN>;
+    using C = Cfg<SPARSE>;
     constexpr int NS = C::STAGES;
-    constexpr int BK = 128 / ELT;                     // logical K per stage (B rows are 128 bytes of K)
-    constexpr int MMA_PER_STAGE = SPARSE ? 2 : 4;     // sparse: 64 B of B's K per instruction, dense: 32 B
     constexpr bool F8 = (ELT == 1);
+    constexpr int BK = (SPARSE ? 256 : 128) / ELT;    // logical K per stage
+    constexpr int B_SUBS = SPARSE ? 2 : 1;
+    constexpr int SUB_K = 128 / ELT;                  // logical K of one B sub-tile
+    constexpr int ATOMS_PER_STAGE = SPARSE ? BK / 128 : 1;   // metadata atoms (128 logical K) per stage
     constexpr int B_CHUNK_N = 128 / ELT;              // MN-major: N elements per 128-byte row
-    constexpr int B_CHUNKS = BN / B_CHUNK_N;
+    constexpr int B_CHUNKS_HALF = (BN / 2) / B_CHUNK_N;
+    constexpr uint32_t STAGE_TX = 2u * C::STAGE;      // both CTAs' operand bytes
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bars = smem_base + NS * C::STAGE;             // barrier block, 8-byte aligned
-    auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (NS + s); };
-    auto acc_full_bar = [&](int b) { return bars + 8u * (2 * NS + b); };
-    auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * NS + 2 + b); };
-    const uint32_t tmem_slot = bars + 8u * (2 * NS + 4);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_raw + (bars - smem_u32(smem_raw)) + 8u * (2 * NS + 5));
-    volatile uint32_t *tmem_slot_ptr =
-        reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+    const uint32_t staging = smem_base + NS * C::STAGE;
+    const uint32_t bars = staging + STAGING_BYTES;
+    auto full_bar = [&](int s) { return bars + 8u * s; };              // used in the leader only
+    auto empty_bar = [&](int s) { return bars + 8u * (NS + s); };      // one per CTA
+    const uint32_t acc_full_bar = bars + 8u * (2 * NS);                // one per CTA
+    const uint32_t acc_empty_bar = bars + 8u * (2 * NS + 1);           // leader only, 2 arrivals
+    auto meta_full_bar = [&](int r) { return bars + 8u * (2 * NS + 2 + r); };             // leader only, 8 arrivals
+    auto meta_empty_bar = [&](int r) { return bars + 8u * (2 * NS + 2 + META_REGIONS + r); };   // one per CTA
+    const uint32_t tmem_slot = bars + 8u * (2 * NS + 2 + 2 * META_REGIONS);
+    uint8_t *bars_generic = smem_raw + (bars - smem_u32(smem_raw));
+    volatile uint32_t *tmem_slot_ptr = reinterpret_cast<volatile uint32_t *>(bars_generic + 8u * (2 * NS + 2 + 2 * META_REGIONS));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_generic + 8u * (2 * NS + 3 + 2 * META_REGIONS));
+    uint8_t *staging_generic = smem_raw + (staging - smem_u32(smem_raw));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m_tiles = p.M / BM;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = (rank == 0);
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM);
     const int n_tiles = (p.N + BN - 1) / BN;
     const int num_tiles = m_tiles * n_tiles;
-    const int k_blocks = p.K / BK;
+    const int k_blocks = (p.K + BK - 1) / BK;         // a ragged last stage reads zero-filled K
+    const int k_atoms = p.K / 128;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 4); }
+        mbar_init(acc_full_bar, 1);
+        mbar_init(acc_empty_bar, 2);
+        for (int r = 0; r < META_REGIONS; ++r) { mbar_init(meta_full_bar(r), 8); mbar_init(meta_empty_bar(r), 1); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
+        if (!OUT_F32) prefetch_tensormap(&map_d);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, TMEM_COLS);
@@ -234,174 +319,294 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync();          // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
                 const int mt = tile % m_tiles, nt = tile / m_tiles;
+                const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;      // this CTA's rows of A
+                const int n0 = nt * BN + static_cast<int>(rank) * (BN / 2);    // this CTA's half of B
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1u;
+                    if (PROBE_MODE(p) == 3 && it >= static_cast<uint32_t>(NS)) continue;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, p.status, abort_flag)) { ok = false; break; }
+                    const uint32_t lead_full = map_to_cta(full_bar(s), 0);
+                    if (PROBE_MODE(p) == 1 && it >= static_cast<uint32_t>(NS)) {
+                        if (leader) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full_bar(s)) : "memory");
+                        continue;
+                    }
+                    if (leader) mbar_arrive_expect_tx(full_bar(s), STAGE_TX);
                     const uint32_t a_dst = smem_base + s * C::STAGE;
                     const uint32_t b_dst = a_dst + C::A_STAGE;
-                    const bool load_meta = SPARSE && (F8 || (kb & 1) == 0);
-                    mbar_arrive_expect_tx(full_bar(s), C::A_STAGE + C::B_STAGE + (load_meta ? 2048u : 0u));
-                    // A: rows mt*128.., 64 bytes (compressed) or 128 bytes of K per row
-                    tma_load_2d(a_dst, &map_a, full_bar(s), kb * (SPARSE ? BK / 2 : BK), mt * BM);
-                    if (BMAJ == BMajor::K) {
-                        tma_load_2d(b_dst, &map_b, full_bar(s), kb * BK, nt * BN);
-                    } else {
+                    // A: 128 bytes per row = BK/2 compressed (sparse) or BK dense elements
+                    tma_load_2d(a_dst, &map_a, lead_full, kb * (SPARSE ? BK / 2 : BK), m0);
 #pragma unroll
-                        for (int c = 0; c < B_CHUNKS; ++c)
-                            tma_load_2d(b_dst + c * (BK * 128), &map_b, full_bar(s), nt * BN + c * B_CHUNK_N, kb * BK);
-                    }
-                    if (load_meta) {
-                        const int atom_k = F8 ? kb : (kb >> 1);
-                        const size_t atom = static_cast<size_t>(mt) * (p.K / 128) + atom_k;
-                        bulk_load(b_dst + C::B_STAGE, p.meta + atom * 2048, 2048, full_bar(s));
+                    for (int u = 0; u < B_SUBS; ++u) {
+                        const int k0 = kb * BK + u * SUB_K;
+                        if (BMAJ == BMajor::K) {
+                            tma_load_2d(b_dst + u * C::B_SUB, &map_b, lead_full, k0, n0);
+                        } else if (SPARSE) {
+                            // MN-major: one box per 128-byte N chunk spans the whole stage's K rows
+                            if (u == 0) {
+#pragma unroll
+                                for (int c = 0; c < B_CHUNKS_HALF; ++c)
+                                    tma_load_2d(b_dst + c * (BK * 128), &map_b, lead_full, n0 + c * B_CHUNK_N, kb * BK);
+                            }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < B_CHUNKS_HALF; ++c)
+                                tma_load_2d(b_dst + c * (BK * 128), &map_b, lead_full, n0 + c * B_CHUNK_N, kb * BK);
+                        }
                     }
                 }
             }
-            if (!ok) {
-                // give copies already in flight time to land before the CTA leaves (bounded)
-                const long long start = clock64();
-                while (clock64() - start < 4000000ll) { }
-            }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc(SPARSE, p.afmt, p.bfmt, BMAJ == BMajor::MN, BN);
-            uint32_t it = 0, local_tile = 0;
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (leader && lane == 0) {
+            const uint32_t idesc = instr_desc(SPARSE, p.afmt, p.bfmt, BMAJ == BMajor::MN);
+            uint32_t it = 0, local_tile = 0, group_it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local_tile) {
-                const int buf = (C::ACC_BUFS == 2) ? (local_tile & 1) : 0;
-                const uint32_t use = (C::ACC_BUFS == 2) ? (local_tile >> 1) : local_tile;
-                if (!mbar_wait(acc_empty_bar(buf), (use & 1u) ^ 1u, p.status, abort_flag)) { ok = false; break; }
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++local_tile) {
+                if (!mbar_wait(acc_empty_bar, (local_tile & 1u) ^ 1u, p.status, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * BN;
+                PROBE_STAMP(p, local_tile, 0);
+                const uint32_t d_tmem = tmem_base;
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1u;
-                    if (!mbar_wait(full_bar(s), ph, p.status, abort_flag)) { ok = false; break; }
+                    uint32_t meta_cols = 0;
+                    if (SPARSE) {
+                        // metadata groups of four atoms rotate over META_REGIONS tensor-memory regions,
+                        // written by the metadata warps of both CTAs
+                        const int atom0 = kb * ATOMS_PER_STAGE;
+                        const uint32_t region = group_it % META_REGIONS;
+                        if ((atom0 & 3) == 0 &&
+                            !mbar_wait(meta_full_bar(region), (group_it / META_REGIONS) & 1u, p.status, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        meta_cols = tmem_base + META_COL0 + 16 * region + 4 * (atom0 & 3);
+                    }
+                    if (!(PROBE_MODE(p) == 3 && it >= static_cast<uint32_t>(NS)) &&
+                        !mbar_wait(full_bar(s), ph, p.status, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_src = smem_base + s * C::STAGE;
                     const uint32_t b_src = a_src + C::A_STAGE;
-                    uint32_t e_tmem = 0;
-                    if (SPARSE) {
-                        // One metadata atom (128 logical K, four 32-bit columns) per stage for fp8 and per two
-                        // stages for bf16 (it arrives with the even k-block).  Tensor-memory regions rotate
-                        // over NS atoms, so a region is rewritten only after the stages that read it retired.
-                        const uint32_t atom_it = F8 ? it : (it >> 1);
-                        const uint32_t region = tmem_base + C::META_COL0 + 4 * (atom_it % NS);
-                        if (F8 || (kb & 1) == 0) {
-                            const uint64_t mdesc = smem_desc(b_src + C::B_STAGE, 16, 128, 0);
-                            tc_cp_128x128b(region, mdesc);
-                        }
-                        e_tmem = region + ((!F8 && (kb & 1)) ? 2u : 0u);
-                    }
 #pragma unroll
-                    for (int j = 0; j < MMA_PER_STAGE; ++j) {
-                        const uint64_t adesc = SPARSE ? smem_desc(a_src + 32 * j, 16, 512, 4)
-                                                      : smem_desc(a_src + 32 * j, 16, 1024, 2);
+                    for (int j = 0; j < 4; ++j) {
+                        if (PROBE_MODE(p) == 2) break;
+                        const uint64_t adesc = smem_desc(a_src + 32 * j, 16, 1024, 2);
                         uint64_t bdesc;
                         if (BMAJ == BMajor::K) {
-                            bdesc = smem_desc(b_src + (SPARSE ? 64 : 32) * j, 16, 1024, 2);
+                            bdesc = SPARSE ? smem_desc(b_src + (j >> 1) * C::B_SUB + 64 * (j & 1), 16, 1024, 2)
+                                           : smem_desc(b_src + 32 * j, 16, 1024, 2);
                         } else {
-                            constexpr int ROWS_PER_MMA = BK / MMA_PER_STAGE;     // K rows of 128 bytes per instruction
+                            constexpr int ROWS_PER_MMA = BK / 4;     // K rows of 128 bytes per instruction
                             bdesc = smem_desc(b_src + ROWS_PER_MMA * 128 * j, BK * 128, 1024, 2);
                         }
                         const uint32_t acc = (kb > 0 || j > 0) ? 1u : 0u;
                         if (SPARSE) {
-                            // bf16: one 32-bit metadata column per instruction, pairs selected by the descriptor's
-                            // sparse selector; fp8: two columns per instruction
-                            const uint32_t e = F8 ? (e_tmem + 2 * j) : e_tmem;
-                            const uint32_t id2 = F8 ? 0u : static_cast<uint32_t>(j);
+                            // bf16: one 32-bit metadata column per instruction, the column pair is addressed and
+                            // the descriptor's sparse selector picks the column; fp8: two columns per instruction
+                            const uint32_t e = meta_cols + (F8 ? 2 * j : (j & 2));
+                            const uint32_t id2 = F8 ? 0u : static_cast<uint32_t>(j & 1);
                             tc_mma_sparse<F8>(d_tmem, adesc, bdesc, e, idesc | id2, acc);
                         } else {
                             tc_mma_dense<F8>(d_tmem, adesc, bdesc, idesc, acc);
                         }
                     }
-                    tc_commit(empty_bar(s));     // frees the stage once these MMAs (and the cp) have read it
-                }
-                if (ok) tc_commit(acc_full_bar(buf));
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5)
-        const int quarter = warp & 3;                  // tensor-memory lanes [32*quarter, 32*quarter + 32)
-        const float scale = p.out_scale ? *p.out_scale : 1.0f;
-        uint32_t local_tile = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local_tile) {
-            const int mt = tile % m_tiles, nt = tile / m_tiles;
-            const int buf = (C::ACC_BUFS == 2) ? (local_tile & 1) : 0;
-            const uint32_t use = (C::ACC_BUFS == 2) ? (local_tile >> 1) : local_tile;
-            if (!mbar_wait(acc_full_bar(buf), use & 1u, p.status, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const int m = mt * BM + quarter * 32 + lane;
-            const int n_valid = min(BN, p.N - nt * BN);
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (c0 >= n_valid) break;
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * BN + c0, r);
-                tmem_ld_wait();
-                const int n0 = nt * BN + c0;
-                if (OUT_T) {
-                    // out[n, m]: 32 lanes write 32 consecutive m for each n
-                    if (OUT_F32) {
-                        float *out = static_cast<float *>(p.D);
-#pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            out[static_cast<size_t>(n0 + c) * p.M + m] = __fmul_rn(__uint_as_float(r[c]), scale);
-                    } else {
-                        __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(p.D);
-#pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            out[static_cast<size_t>(n0 + c) * p.M + m] =
-                                __float2bfloat16_rn(__fmul_rn(__uint_as_float(r[c]), scale));
-                    }
-                } else {
-                    if (OUT_F32) {
-                        float4 *out = reinterpret_cast<float4 *>(static_cast<float *>(p.D) + static_cast<size_t>(m) * p.N + n0);
-#pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            out[c] = make_float4(__fmul_rn(__uint_as_float(r[4 * c]), scale),
-                                                 __fmul_rn(__uint_as_float(r[4 * c + 1]), scale),
-                                                 __fmul_rn(__uint_as_float(r[4 * c + 2]), scale),
-                                                 __fmul_rn(__uint_as_float(r[4 * c + 3]), scale));
-                    } else {
-                        uint4 *out = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.D) + static_cast<size_t>(m) * p.N + n0);
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float lo = __fmul_rn(__uint_as_float(r[8 * c + 2 * e]), scale);
-                                const float hi = __fmul_rn(__uint_as_float(r[8 * c + 2 * e + 1]), scale);
-                                w[e] = sste_f32_to_bf16_bits(lo) | (sste_f32_to_bf16_bits(hi) << 16);
-                            }
-                            out[c] = make_uint4(w[0], w[1], w[2], w[3]);
+                    tc_commit_pair(empty_bar(s));     // frees the stage in both CTAs once these MMAs have read it
+                    if (SPARSE) {
+                        const int atom_end = (kb + 1) * ATOMS_PER_STAGE;
+                        if ((atom_end & 3) == 0 || kb == k_blocks - 1) {
+                            tc_commit_pair(meta_empty_bar(group_it % META_REGIONS));
+                            ++group_it;
                         }
                     }
                 }
+                if (ok) tc_commit_pair(acc_full_bar);
+                PROBE_STAMP(p, local_tile, 1);
             }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        const int quarter = warp & 3;                  // tensor-memory lanes [32*quarter, 32*quarter + 32)
+        const int row = quarter * 32 + lane;           // row of this CTA's 128 x BN accumulator
+        const float scale = p.out_scale ? *p.out_scale : 1.0f;
+        const bool store_thread = (threadIdx.x == 64);
+        const uint32_t lead_acc_empty = map_to_cta(acc_empty_bar, 0);
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        uint32_t local_tile = 0;
+        bool ok = true;
+        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++local_tile) {
+            const int mt = tile % m_tiles, nt = tile / m_tiles;
+            const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;
+            const int n0 = nt * BN;
+            if (!mbar_wait_warp(acc_full_bar, local_tile & 1u, p.status, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            if (threadIdx.x == 64) PROBE_STAMP(p, local_tile, 2);
+            if (OUT_F32) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(lane_base + c0, r);
+                    tmem_ld_wait();
+                    const int m = m0 + row;
+                    if (m < p.M && n0 + c0 < p.N) {
+                        if (OUT_T) {
+                            float *out = static_cast<float *>(p.D);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                out[static_cast<size_t>(n0 + c0 + c) * p.M + m] = __fmul_rn(__uint_as_float(r[c]), scale);
+                        } else {
+                            float4 *out = reinterpret_cast<float4 *>(static_cast<float *>(p.D) +
+                                                                     static_cast<size_t>(m) * p.N + n0 + c0);
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                out[c] = make_float4(__fmul_rn(__uint_as_float(r[4 * c]), scale),
+                                                     __fmul_rn(__uint_as_float(r[4 * c + 1]), scale),
+                                                     __fmul_rn(__uint_as_float(r[4 * c + 2]), scale),
+                                                     __fmul_rn(__uint_as_float(r[4 * c + 3]), scale));
+                        }
+                    }
+                }
+                tc_fence_before();
+                epilogue_barrier();
+                if (store_thread) {
+                    PROBE_STAMP(p, local_tile, 3);
+                    mbar_arrive_cluster(lead_acc_empty);
+                }
+                continue;
+            }
+            // bf16 output: two passes of 128 columns through a 32 KB staging buffer and TMA stores.
+            // The second half is pulled into registers first, so the accumulator is released before
+            // its conversion and stores.
+            auto stage_chunk = [&](const uint32_t (&r)[32], int c0 /* column inside the 128-column half */) {
+                if (OUT_T) {
+                    // staging[n][m]: 128 rows of 128 bf16; a warp writes 32 consecutive m per n
+                    uint16_t *st = reinterpret_cast<uint16_t *>(staging_generic);
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        st[(c0 + c) * BM + row] =
+                            static_cast<uint16_t>(sste_f32_to_bf16_bits(__fmul_rn(__uint_as_float(r[c]), scale)));
+                } else {
+                    // two sub-tiles [128 rows][64 bf16] with the 128-byte swizzle of the TMA store:
+                    // 16-byte chunk index ^= row & 7
+                    uint8_t *sub = staging_generic + (c0 >> 6) * 16384 + row * 128;
+                    const int chunk0 = (c0 & 63) >> 3;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float lo = __fmul_rn(__uint_as_float(r[8 * c + 2 * e]), scale);
+                            const float hi = __fmul_rn(__uint_as_float(r[8 * c + 2 * e + 1]), scale);
+                            w[e] = sste_f32_to_bf16_bits(lo) | (sste_f32_to_bf16_bits(hi) << 16);
+                        }
+                        *reinterpret_cast<uint4 *>(sub + (((chunk0 + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            };
+            auto store_half = [&](int half) {
+                if (OUT_T) {
+                    tma_store_2d(&map_d, staging, m0, n0 + 128 * half);
+                } else {
+                    tma_store_2d(&map_d, staging, n0 + 128 * half, m0);
+                    tma_store_2d(&map_d, staging + 16384, n0 + 128 * half + 64, m0);
+                }
+                tma_store_commit();
+            };
+            // first half: the previous tile's store must have finished reading the staging buffer
+            if (store_thread) tma_store_wait_read();
+            epilogue_barrier();
+            {
+                uint32_t ra[32], rb[32];
+                tmem_ld_32x32(lane_base + 0, ra);
+                tmem_ld_32x32(lane_base + 32, rb);
+                tmem_ld_wait();
+                stage_chunk(ra, 0);
+                tmem_ld_32x32(lane_base + 64, ra);
+                stage_chunk(rb, 32);
+                tmem_ld_32x32(lane_base + 96, rb);
+                tmem_ld_wait();
+                stage_chunk(ra, 64);
+                stage_chunk(rb, 96);
+            }
+            fence_proxy_async();
+            epilogue_barrier();
+            if (store_thread) store_half(0);
+            // second half -> registers, then the accumulator is free
+            uint32_t r0[32], r1[32], r2[32], r3[32];
+            tmem_ld_32x32(lane_base + 128, r0);
+            tmem_ld_32x32(lane_base + 160, r1);
+            tmem_ld_32x32(lane_base + 192, r2);
+            tmem_ld_32x32(lane_base + 224, r3);
+            tmem_ld_wait();
             tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+            if (store_thread) tma_store_wait_read();
+            epilogue_barrier();
+            if (store_thread) {
+                PROBE_STAMP(p, local_tile, 3);
+                mbar_arrive_cluster(lead_acc_empty);
+            }
+            stage_chunk(r0, 0);
+            stage_chunk(r1, 32);
+            stage_chunk(r2, 64);
+            stage_chunk(r3, 96);
+            fence_proxy_async();
+            epilogue_barrier();
+            if (store_thread) store_half(1);
+        }
+        if (store_thread && !OUT_F32) tma_store_wait_all();
+    } else if (SPARSE) {
+        // ------------------------------------------------------------ metadata warps (6..9, both CTAs)
+        // HBM -> registers -> tensor memory: lane L of an atom's image is exactly the 16 bytes the
+        // instruction expects in tensor-memory lane L, four 32-bit columns per atom.
+        const int quarter = warp & 3;
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + META_COL0;
+        uint32_t group_it = 0;
+        bool ok = true;
+        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            const int mt = tile % m_tiles;
+            const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;
+            const bool rows_valid = m0 < p.M;
+            const uint4 *src = reinterpret_cast<const uint4 *>(meta + static_cast<size_t>(m0 / BM) * k_atoms * 2048) +
+                               quarter * 32 + lane;
+            const int atoms_padded = k_blocks * ATOMS_PER_STAGE;
+            for (int a0 = 0; a0 < atoms_padded; a0 += 4, ++group_it) {
+                const uint32_t region = group_it % META_REGIONS;
+                if (!mbar_wait_warp(meta_empty_bar(region), ((group_it / META_REGIONS) & 1u) ^ 1u, p.status, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                uint4 v[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    v[i] = (rows_valid && a0 + i < k_atoms) ? __ldg(src + static_cast<size_t>(a0 + i) * 128)
+                                                            : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) tmem_st_32x4(lane_base + 16 * region + 4 * i, v[i]);
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(meta_full_bar(region), 0));
+            }
         }
     }
 
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    cluster_sync();          // neither CTA frees tensor memory while the pair still uses it
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
@@ -428,33 +633,46 @@ bool make_map(const sste_ctx *ctx, CUtensorMap *map, const void *base, int elt, 
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32>
-sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const GemmParams &p, cudaStream_t stream)
+template <bool SPARSE, BMajor BMAJ, int ELT, bool OUT_T, bool OUT_F32>
+sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void *meta, const GemmParams &p,
+                   cudaStream_t stream)
 {
-    using C = Cfg<SPARSE, BN>;
-    constexpr int BK = 128 / ELT;
-    CUtensorMap map_a, map_b;
+    using C = Cfg<SPARSE>;
+    constexpr int BK = (SPARSE ? 256 : 128) / ELT;
+    CUtensorMap map_a, map_b, map_d;
     bool ok;
-    if (SPARSE)   // compressed values [M, K/2], 64 bytes of K per row per stage
-        ok = make_map(ctx, &map_a, A, ELT, p.M, p.K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (SPARSE)   // compressed values [M, K/2]: 128 bytes per row per stage
+        ok = make_map(ctx, &map_a, A, ELT, p.M, p.K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_128B);
     else
         ok = make_map(ctx, &map_a, A, ELT, p.M, p.K, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B);
-    if (BMAJ == BMajor::K)   // B stored [N, K]
-        ok = ok && make_map(ctx, &map_b, B, ELT, p.N, p.K, BK, BN, CU_TENSOR_MAP_SWIZZLE_128B);
-    else                     // B stored [K, N]
+    if (BMAJ == BMajor::K)   // B stored [N, K]: sub-tiles of BN/2 rows by 128 bytes of K
+        ok = ok && make_map(ctx, &map_b, B, ELT, p.N, p.K, 128 / ELT, BN / 2, CU_TENSOR_MAP_SWIZZLE_128B);
+    else                     // B stored [K, N]: chunks of 128 bytes of N by BK rows of K
         ok = ok && make_map(ctx, &map_b, B, ELT, p.K, p.N, 128 / ELT, BK, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (OUT_F32) {
+        map_d = map_a;       // unused: the fp32 epilogue stores directly
+    } else if (OUT_T) {      // out[N, M] bf16: box = 128 m x 128 n
+        ok = ok && make_map(ctx, &map_d, p.D, 2, p.N, p.M, BM, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+    } else {                 // out[M, N] bf16: boxes of 64 n x 128 m, 128-byte swizzle
+        ok = ok && make_map(ctx, &map_d, p.D, 2, p.M, p.N, 64, BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    }
     if (!ok) return SSTE_ERR_CUDA;
-    auto kern = gemm_kernel<SPARSE, BMAJ, ELT, BN, OUT_T, OUT_F32>;
+    auto kern = gemm_kernel<SPARSE, BMAJ, ELT, OUT_T, OUT_F32>;
     static bool attr_set = false;   // per instantiation
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
             return SSTE_ERR_CUDA;
         attr_set = true;
     }
-    const int m_tiles = p.M / BM, n_tiles = (p.N + BN - 1) / BN;
-    int grid = m_tiles * n_tiles;
-    if (grid > ctx->sm_count) grid = ctx->sm_count;
-    kern<<<grid, GEMM_THREADS, C::SMEM_BYTES, stream>>>(map_a, map_b, p);
+    const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM), n_tiles = (p.N + BN - 1) / BN;
+    int pairs = m_tiles * n_tiles;
+    if (pairs > ctx->sm_count / 2) pairs = ctx->sm_count / 2;
+    GemmParams pp = p;
+#ifdef SSTE_PROBE
+    pp.probe = g_probe_mode;
+    pp.dbg = g_probe_dbg;
+#endif
+    kern<<<2 * pairs, C::THREADS, C::SMEM_BYTES, stream>>>(map_a, map_b, map_d, static_cast<const uint8_t *>(meta), pp);
     return cudaGetLastError() == cudaSuccess ? SSTE_OK : SSTE_ERR_CUDA;
 }
 
@@ -469,18 +687,22 @@ bool fmt_code(sste_dtype dt, int *elt, uint32_t *code)
 }
 
 // dispatch on output dtype
-template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T>
-sste_status launch_out(const sste_ctx *ctx, const void *A, const void *B, const GemmParams &p, sste_dtype odt,
-                       cudaStream_t s)
+template <bool SPARSE, BMajor BMAJ, int ELT, bool OUT_T>
+sste_status launch_out(const sste_ctx *ctx, const void *A, const void *B, const void *meta, const GemmParams &p,
+                       sste_dtype odt, cudaStream_t s)
 {
-    if (odt == SSTE_F32) return launch<SPARSE, BMAJ, ELT, BN, OUT_T, true>(ctx, A, B, p, s);
-    if (odt == SSTE_BF16) return launch<SPARSE, BMAJ, ELT, BN, OUT_T, false>(ctx, A, B, p, s);
+    if (odt == SSTE_F32) return launch<SPARSE, BMAJ, ELT, OUT_T, true>(ctx, A, B, meta, p, s);
+    if (odt == SSTE_BF16) return launch<SPARSE, BMAJ, ELT, OUT_T, false>(ctx, A, B, meta, p, s);
     return SSTE_ERR_DTYPE;
 }
 
 }  // namespace
 
 sste_status sste_gemm_launch_check(const sste_ctx *) { return SSTE_OK; }
+#ifdef SSTE_PROBE
+extern "C" void sste_probe_set_mode(int mode) { g_probe_mode = mode; }
+extern "C" void sste_probe_set_dbg(long long *dbg) { g_probe_dbg = dbg; }
+#endif
 
 extern "C" sste_status sste_linear_fwd(sste_ctx *ctx, const void *X, int T, const void *vals, const void *meta, int O,
                                        int I, sste_dtype opdt, const float *out_scale_dev, void *Y, sste_dtype ydt,
@@ -497,10 +719,10 @@ extern "C" sste_status sste_linear_fwd(sste_ctx *ctx, const void *X, int T, cons
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
     // Z^T[O, T] = S(W)[O, I] X^T: M = O, N = T, K = I; the output is stored transposed as Y[T, O]
-    GemmParams p{O, T, I, static_cast<const uint8_t *>(meta), Y, out_scale_dev, ctx->status_dev, code, code};
+    GemmParams p{O, T, I, Y, out_scale_dev, ctx->status_dev, code, code};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (elt == 2) return launch_out<true, BMajor::K, 2, 256, true>(ctx, vals, X, p, ydt, s);
-    return launch_out<true, BMajor::K, 1, 256, true>(ctx, vals, X, p, ydt, s);
+    if (elt == 2) return launch_out<true, BMajor::K, 2, true>(ctx, vals, X, meta, p, ydt, s);
+    return launch_out<true, BMajor::K, 1, true>(ctx, vals, X, meta, p, ydt, s);
 }
 
 extern "C" sste_status sste_linear_bwd_weight(sste_ctx *ctx, const void *gvals, const void *gmeta, int O, int T,
@@ -519,10 +741,10 @@ extern "C" sste_status sste_linear_bwd_weight(sste_ctx *ctx, const void *gvals, 
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
     // grad_W[O, I] = G[O, T] X[T, I]: M = O, N = I, K = T; X is [K, N] row-major = MN-major B
-    GemmParams p{O, I, T, static_cast<const uint8_t *>(gmeta), dW, out_scale_dev, ctx->status_dev, ca, cb};
+    GemmParams p{O, I, T, dW, out_scale_dev, ctx->status_dev, ca, cb};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (ea == 2) return launch_out<true, BMajor::MN, 2, 256, false>(ctx, gvals, X, p, dwdt, s);
-    return launch_out<true, BMajor::MN, 1, 256, false>(ctx, gvals, X, p, dwdt, s);
+    if (ea == 2) return launch_out<true, BMajor::MN, 2, false>(ctx, gvals, X, gmeta, p, dwdt, s);
+    return launch_out<true, BMajor::MN, 1, false>(ctx, gvals, X, gmeta, p, dwdt, s);
 }
 
 extern "C" sste_status sste_linear_bwd_input(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt,
@@ -540,8 +762,8 @@ extern "C" sste_status sste_linear_bwd_input(sste_ctx *ctx, const void *dY, int 
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
     // grad_X[T, I] = grad_Z[T, O] S(W)[O, I]: M = T, N = I, K = O; S(W) is [K, N] row-major = MN-major B
-    GemmParams p{T, I, O, nullptr, dX, out_scale_dev, ctx->status_dev, ca, cb};
+    GemmParams p{T, I, O, dX, out_scale_dev, ctx->status_dev, ca, cb};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (ea == 2) return launch_out<false, BMajor::MN, 2, 256, false>(ctx, dY, Wt_dense, p, xdt, s);
-    return launch_out<false, BMajor::MN, 1, 256, false>(ctx, dY, Wt_dense, p, xdt, s);
+    if (ea == 2) return launch_out<false, BMajor::MN, 2, false>(ctx, dY, Wt_dense, nullptr, p, xdt, s);
+    return launch_out<false, BMajor::MN, 1, false>(ctx, dY, Wt_dense, nullptr, p, xdt, s);
 }
