@@ -152,7 +152,7 @@ def workload_config(cfg_id, cfg, n_gpus):
     return {"workload": f"BASELINE config {cfg_id}: " + ", ".join(f"{L.name} W[{L.O},{L.I}] x {L.T} tokens" for L in cfg["layers"]),
             "precision": "fp8 (e4m3 fwd / e5m2 bwd)" if cfg["fp8"] else "bf16",
             "tokens_per_gpu": cfg["layers"][0].T, "parallelism": f"dp{n_gpus} (token shards, no data-path collective)",
-            "l2": "flushed between timed steps (512 MiB write)"}
+            "l2": "flushed between timed steps (512 MiB write)", "launch": "one CUDA-graph replay per step"}
 
 
 # --------------------------------------------------------------------------------------------- GPU arm
@@ -229,31 +229,53 @@ def run_gpu(args):
     for w in range(max(args.warmup, 3)):
         step(w)
     barrier()
+
+    # The timed step is one CUDA-graph replay of all launches of the step (no host work between kernels);
+    # the MVUE step counter is frozen in the graph, which does not change the work done.
+    graph = None
+    if not args.no_graph:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step(args.warmup)
+        graph.replay()
+        torch.cuda.synchronize()
     launches_before = sum(l.launches for l, _, _ in layers)
+    launches_per_step = None
 
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
-    per_kernel = {k: [] for k in KERNELS}
     step_ms = []
     barrier()
     for s in range(args.steps):
         flush.zero_()                                   # evict L2 between timed steps
-        ev = []
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        step(args.warmup + s, ev)
+        if graph is not None:
+            graph.replay()
+        else:
+            step(args.warmup + s)
         e1.record(stream)
         torch.cuda.synchronize()
         step_ms.append(e0.elapsed_time(e1))
+    barrier()
+    # second timed pass, eager, with an event between kernels: the per-kernel breakdown and roofline
+    per_kernel = {k: [] for k in KERNELS}
+    n_before = sum(l.launches for l, _, _ in layers)
+    for s in range(args.steps):
+        flush.zero_()
+        ev = []
+        step(args.warmup + s, ev)
+        torch.cuda.synchronize()
         if not fp8:
             for li in range(len(layers)):
                 base = li * 6
                 for ki, k in enumerate(KERNELS):
                     per_kernel[k].append((li, ev[base + ki].elapsed_time(ev[base + ki + 1])))
+    launches_per_step = (sum(l.launches for l, _, _ in layers) - n_before) // args.steps
     barrier()
     clocks = sampler.stop()
-    gpu_launches = sum(l.launches for l, _, _ in layers) - launches_before
+    gpu_launches = launches_per_step * args.steps       # kernels executed inside the timed region
     total_ms = sum(step_ms)
     if world > 1:
         t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
@@ -352,6 +374,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="BASELINE config id (2 = GPT-2-small MLP, the default workload)")
+    ap.add_argument("--no-graph", action="store_true", help="launch the timed steps eagerly instead of replaying a CUDA graph")
     ap.add_argument("--ref-tokens", type=int, default=8192, help="tokens per layer in the CPU-oracle sample")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -70,6 +70,10 @@ typedef enum { SSTE_BF16 = 0, SSTE_F32 = 1, SSTE_E4M3 = 2, SSTE_E5M2 = 3 } sste_
 
 /* Bytes of caller-owned device workspace a context needs (status word + reduction scratch). */
 size_t sste_workspace_bytes(void);
+/* A larger workspace (this many bytes or more) also lets the three products split their reduction
+ * dimension over several CTA pairs when a product has fewer output tiles than the GPU has CTA pairs
+ * (fp32 partial tiles live in the workspace); with the minimal workspace they never split. */
+size_t sste_workspace_bytes_recommended(void);
 
 /*
  * Create a context on `device`.  `workspace` is device memory of at least
@@ -181,6 +185,15 @@ sste_status sste_scalar_mul(sste_ctx *ctx, const float *a_dev, const float *b_de
 /* Operand-image metadata -> canonical uint16 [rows, k/16] (see top).  dt selects the 16-bit or 8-bit image. */
 sste_status sste_meta_to_canonical(sste_ctx *ctx, const void *meta, int rows, int k, sste_dtype dt,
                                    void *canonical_out, void *stream);
+
+/* The three products pick the width of their output tiles (128, 192 or 256 columns) from the problem
+ * shape.  This process-wide hook pins it so that tests can cover every variant; widths a product does
+ * not support (192 needs a K-major B operand, i.e. the forward) fall back to the automatic choice.
+ * bn: 0 (automatic), 128, 192 or 256; anything else gives SSTE_ERR_INVALID_ARG. */
+sste_status sste_debug_force_tile_width(int bn);
+/* Same for the split-K factor: 0 (automatic) or 1..4; a factor the shape or the workspace does not allow
+ * falls back to the automatic choice. */
+sste_status sste_debug_force_splits(int splits);
 
 #ifdef __cplusplus
 }

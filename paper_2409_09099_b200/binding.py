@@ -26,7 +26,8 @@ EXPORTS = [
     "sste_workspace_bytes", "sste_create", "sste_destroy", "sste_status_string", "sste_poll_device_status",
     "sste_vals_bytes", "sste_meta_bytes", "sste_beta_init", "sste_project_compress", "sste_linear_fwd",
     "sste_mvue_sparsify", "sste_linear_bwd_input", "sste_linear_bwd_weight", "sste_amax", "sste_fp8_scale",
-    "sste_quantize_fp8", "sste_scalar_mul", "sste_meta_to_canonical",
+    "sste_quantize_fp8", "sste_scalar_mul", "sste_meta_to_canonical", "sste_debug_force_tile_width", "sste_debug_force_splits",
+    "sste_workspace_bytes_recommended",
 ]
 
 
@@ -47,6 +48,7 @@ def load() -> ctypes.CDLL:
             raise FileNotFoundError(f"{LIB_PATH} not built: run python -m paper_2409_09099_b200.build")
         lib = ctypes.CDLL(str(LIB_PATH))
         lib.sste_workspace_bytes.restype = ctypes.c_size_t
+        lib.sste_workspace_bytes_recommended.restype = ctypes.c_size_t
         lib.sste_vals_bytes.restype = ctypes.c_size_t
         lib.sste_meta_bytes.restype = ctypes.c_size_t
         lib.sste_status_string.restype = ctypes.c_char_p
@@ -68,10 +70,10 @@ def _stream():
 class Context:
     """Owns the device workspace (a torch allocation) and the sste_ctx handle."""
 
-    def __init__(self, device: int = 0):
+    def __init__(self, device: int = 0, minimal_workspace: bool = False):
         self.lib = load()
         self.device = device
-        n = self.lib.sste_workspace_bytes()
+        n = self.lib.sste_workspace_bytes() if minimal_workspace else self.lib.sste_workspace_bytes_recommended()
         self.workspace = torch.zeros(n, dtype=torch.uint8, device=f"cuda:{device}")
         handle = ctypes.c_void_p()
         st = self.lib.sste_create(ctypes.byref(handle), device, _ptr(self.workspace), ctypes.c_size_t(n))
@@ -154,6 +156,12 @@ class Context:
 
     def meta_to_canonical(self, meta, rows, k, dt, out):
         self._check(self.lib.sste_meta_to_canonical(self.handle, _ptr(meta), rows, k, dt, _ptr(out), _stream()))
+
+    def debug_force_splits(self, splits: int):
+        self._check(self.lib.sste_debug_force_splits(splits))
+
+    def debug_force_tile_width(self, bn: int):
+        self._check(self.lib.sste_debug_force_tile_width(bn))
 
     def poll_device_status(self) -> int:
         return self.lib.sste_poll_device_status(self.handle, _stream())

@@ -8,6 +8,8 @@
 namespace {
 
 constexpr int EW_THREADS = 256;
+constexpr int PC_ROWS = 32;                                  // rows of W per project+compress CTA
+constexpr int PC_CHUNKS = PC_ROWS * 16 / EW_THREADS;         // 16-byte chunks per thread
 
 // ---------------------------------------------------------------- group of four: S_soft + kept pair
 
@@ -61,29 +63,31 @@ __device__ __forceinline__ float sel4(uint32_t idx, float v0, float v1, float v2
 
 // ---------------------------------------------------------------- project + compress
 
-// One CTA: 128 rows x 128 input features of W.  Thread = 8 chunks of 8 consecutive features.
+// One CTA: 32 rows x 128 input features of W (a quarter of a metadata atom, 512 contiguous bytes of its
+// image); a thread handles two chunks of 8 consecutive features.  Small tiles keep even the 2.4 M-element
+// GPT-2 weights spread over several CTAs per SM.
 template <bool FP8>
 __global__ void __launch_bounds__(EW_THREADS)
 project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restrict__ beta_dev,
                         const float *__restrict__ wscale_dev, void *__restrict__ vals, uint8_t *__restrict__ meta,
                         void *__restrict__ dense)
 {
-    __shared__ __align__(16) uint8_t meta_s[2048];
+    __shared__ __align__(16) uint8_t meta_s[512];
     const int tid = threadIdx.x;
     const int kb = blockIdx.x, rb = blockIdx.y;
     const float beta = *beta_dev;
     const float wscale = FP8 ? *wscale_dev : 1.0f;
     const size_t row_chunks = static_cast<size_t>(I) / 8;
 
-    uint4 in[8];
+    uint4 in[PC_CHUNKS];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < PC_CHUNKS; ++i) {
         const int c = i * EW_THREADS + tid;
         const int row = c >> 4, kc = c & 15;
-        in[i] = __ldg(W + (static_cast<size_t>(rb) * 128 + row) * row_chunks + kb * 16 + kc);
+        in[i] = __ldg(W + (static_cast<size_t>(rb) * PC_ROWS + row) * row_chunks + kb * 16 + kc);
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < PC_CHUNKS; ++i) {
         const int c = i * EW_THREADS + tid;
         const int row = c >> 4, kc = c & 15;
         const uint32_t raw[4] = {in[i].x, in[i].y, in[i].z, in[i].w};
@@ -111,8 +115,10 @@ project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restr
             mbyte |= (s.p0 | (s.p1 << 2)) << (4 * g);
         }
         const uint32_t k = 8u * kc;
-        meta_s[FP8 ? sste_meta_atom_byte8(row, k) : sste_meta_atom_byte16(row, k)] = static_cast<uint8_t>(mbyte);
-        const size_t grow = static_cast<size_t>(rb) * 128 + row;
+        const uint32_t arow = (rb & 3) * PC_ROWS + row;   // row inside the 128-row atom
+        meta_s[(FP8 ? sste_meta_atom_byte8(arow, k) : sste_meta_atom_byte16(arow, k)) - 512u * (rb & 3)] =
+            static_cast<uint8_t>(mbyte);
+        const size_t grow = static_cast<size_t>(rb) * PC_ROWS + row;
         const size_t chunk = grow * row_chunks + kb * 16 + kc;   // index in units of 8 input features
         if (FP8) {
             reinterpret_cast<uint32_t *>(vals)[chunk] =
@@ -139,9 +145,9 @@ project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restr
         }
     }
     __syncthreads();
-    if (tid < 128) {
-        const size_t atom = static_cast<size_t>(rb) * (I / 128) + kb;
-        reinterpret_cast<uint4 *>(meta + atom * 2048)[tid] = reinterpret_cast<const uint4 *>(meta_s)[tid];
+    if (tid < 32) {
+        const size_t atom = static_cast<size_t>(rb >> 2) * (I / 128) + kb;
+        reinterpret_cast<uint4 *>(meta + atom * 2048 + 512 * (rb & 3))[tid] = reinterpret_cast<const uint4 *>(meta_s)[tid];
     }
 }
 
@@ -252,53 +258,62 @@ struct MvueGroup {
     float v0, v1;     // their values before the cast
 };
 
+// Inclusion probabilities p_i = min(1, c |a_i|) with sum 2, kept values a_i / p_i, systematic sampling
+// with one uniform u.  With x the first largest magnitude and rest the sum of the others:
+//   clipped   (m_x >= rest): x is kept as is; one other element j, chosen with probability m_j / rest
+//                            by the point u*rest on the others' cumulative sums, carries sign(a_j)*rest;
+//   unclipped (m_x <  rest): the points u*S/2 and u*S/2 + S/2 on the cumulative sums pick two elements,
+//                            both carry sign(a_j)*S/2.
+// Written with one-hot predicates and counting compares instead of index-driven selects (the kernel is
+// bound by the integer/fp32 pipes, not by HBM); every fp32 step is a single rounded operation.
 __device__ __forceinline__ MvueGroup mvue_group(float a0, float a1, float a2, float a3, float u)
 {
     const float m0 = fabsf(a0), m1 = fabsf(a1), m2 = fabsf(a2), m3 = fabsf(a3);
-    uint32_t x = 0;
-    float mx = m0;
-    if (m1 > mx) { x = 1; mx = m1; }
-    if (m2 > mx) { x = 2; mx = m2; }
-    if (m3 > mx) { x = 3; mx = m3; }
-    const uint32_t o0 = (x == 0) ? 1u : 0u, o1 = (x <= 1) ? 2u : 1u, o2 = (x <= 2) ? 3u : 2u;
-    const float mo0 = sel4(o0, m0, m1, m2, m3), mo1 = sel4(o1, m0, m1, m2, m3), mo2 = sel4(o2, m0, m1, m2, m3);
-    const float rest = __fadd_rn(__fadd_rn(mo0, mo1), mo2);
-    uint32_t ja, jb;
-    float va, vb;
-    if (mx >= rest) {
-        // clipped: the largest element is kept with probability 1
-        uint32_t second = o0;
-        float val = 0.0f;
-        if (rest != 0.0f) {
-            const float r = __fmul_rn(u, rest);
-            const float c0 = mo0;
-            const float c1 = __fadd_rn(c0, mo1);
-            second = (c0 > r) ? o0 : (c1 > r) ? o1 : o2;
-            float msec = (c0 > r) ? mo0 : (c1 > r) ? mo1 : mo2;
-            if (msec == 0.0f) second = (mo2 > 0.0f) ? o2 : (mo1 > 0.0f) ? o1 : o0;
-            val = copysignf(rest, sel4(second, a0, a1, a2, a3));
-        }
-        ja = x; va = sel4(x, a0, a1, a2, a3);
-        jb = second; vb = val;
+    const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+    const bool e0 = (m0 == mx);
+    const bool e1 = !e0 && (m1 == mx);
+    const bool e2 = !e0 && !e1 && (m2 == mx);
+    const bool e3 = !e0 && !e1 && !e2;
+    const uint32_t xi = e0 ? 0u : e1 ? 1u : e2 ? 2u : 3u;
+    const float ax = e0 ? a0 : e1 ? a1 : e2 ? a2 : a3;
+    // cumulative sums without x (adding +0 is exact) and with it
+    const float z0 = e0 ? 0.0f : m0;
+    const float z1 = __fadd_rn(z0, e1 ? 0.0f : m1);
+    const float z2 = __fadd_rn(z1, e2 ? 0.0f : m2);
+    const float rest = __fadd_rn(z2, e3 ? 0.0f : m3);
+    const float s1 = __fadd_rn(m0, m1);
+    const float s2 = __fadd_rn(s1, m2);
+    const float s3 = __fadd_rn(s2, m3);
+    const bool clipped = (mx >= rest);
+    const float h = clipped ? rest : __fmul_rn(0.5f, s3);
+    const float c0 = clipped ? z0 : m0, c1 = clipped ? z1 : s1, c2 = clipped ? z2 : s2;
+    const float r1 = __fmul_rn(u, h);
+    const float r2 = __fadd_rn(r1, h);
+    const uint32_t j1 = (c0 <= r1 ? 1u : 0u) + (c1 <= r1 ? 1u : 0u) + (c2 <= r1 ? 1u : 0u);
+    const uint32_t n2 = (c0 <= r2 ? 1u : 0u) + (c1 <= r2 ? 1u : 0u) + (c2 <= r2 ? 1u : 0u);
+    // index pair before ordering: (ia, ib) = (other, x) when clipped, (j1, j2) otherwise
+    uint32_t ia, ib;
+    if (clipped) {
+        ia = (rest == 0.0f) ? (e0 ? 1u : 0u) : j1;
+        ib = xi;
     } else {
-        const float c0 = m0;
-        const float c1 = __fadd_rn(c0, m1);
-        const float c2 = __fadd_rn(c1, m2);
-        const float c3 = __fadd_rn(c2, m3);
-        const float half = __fmul_rn(0.5f, c3);
-        const float r1 = __fmul_rn(u, half);
-        const float r2 = __fadd_rn(r1, half);
-        uint32_t j1 = (c0 > r1) ? 0u : (c1 > r1) ? 1u : (c2 > r1) ? 2u : 3u;
-        uint32_t j2 = 3u;
-        if (j1 < 1u && c1 > r2) j2 = 1u;
-        else if (j1 < 2u && c2 > r2) j2 = 2u;
-        if (j1 == 3u) { j1 = 2u; j2 = 3u; }
-        ja = j1; va = copysignf(half, sel4(j1, a0, a1, a2, a3));
-        jb = j2; vb = copysignf(half, sel4(j2, a0, a1, a2, a3));
+        const bool tail = (j1 == 3u);
+        ia = tail ? 2u : j1;
+        ib = tail ? 3u : max(j1 + 1u, n2);
     }
+    // candidates sign(a_i) * h; a zero h yields +0
+    const uint32_t hb = __float_as_uint(h);
+    const uint32_t sgn = (hb == 0u) ? 0u : 0x80000000u;
+    const float h0 = __uint_as_float((__float_as_uint(a0) & sgn) | hb), h1 = __uint_as_float((__float_as_uint(a1) & sgn) | hb);
+    const float h2 = __uint_as_float((__float_as_uint(a2) & sgn) | hb), h3 = __uint_as_float((__float_as_uint(a3) & sgn) | hb);
+    const float va = sel4(ia, h0, h1, h2, h3);
+    const float vb = clipped ? ax : sel4(ib, h0, h1, h2, h3);
     MvueGroup r;
-    if (ja < jb) { r.q0 = ja; r.v0 = va; r.q1 = jb; r.v1 = vb; }
-    else         { r.q0 = jb; r.v0 = vb; r.q1 = ja; r.v1 = va; }
+    const bool swap = ia > ib;
+    r.q0 = swap ? ib : ia;
+    r.q1 = swap ? ia : ib;
+    r.v0 = swap ? vb : va;
+    r.v1 = swap ? va : vb;
     return r;
 }
 
@@ -533,7 +548,7 @@ extern "C" sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O
         return SSTE_ERR_ALIGN;
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
-    const dim3 grid(I / 128, O / 128);
+    const dim3 grid(I / 128, O / PC_ROWS);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (odt == SSTE_E4M3)
         project_compress_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(W), I, beta_dev,

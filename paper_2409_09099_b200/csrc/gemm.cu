@@ -21,11 +21,9 @@
 namespace {
 
 constexpr int BM = 128;            // rows of A per CTA (a pair covers 256)
-constexpr int BN = 256;            // columns per tile (each CTA stages BN/2 of B)
 constexpr int TMEM_COLS = 512;
-constexpr int META_COL0 = 256;     // accumulators occupy tensor-memory columns [0, 256)
 constexpr int META_REGIONS = 8;   // metadata regions of 16 columns (four atoms) after the accumulators
-constexpr int STAGING_BYTES = 32768;   // half of one CTA's bf16 output tile: 128 x 128 x 2
+constexpr int STAGING_BYTES = 32768;   // two epilogue panels of 128 x 64 bf16
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
 
 enum class BMajor { K, MN };
@@ -207,10 +205,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 // Instruction descriptor: sparse selector [0,2), sparse flag [2], D = fp32 [4,6), A format [7,10),
 // B format [10,13), A major [15], B major [16] (1 = MN-major), N>>3 [17,23), M>>4 [24,29).
 // M is 256: the pair's two 128-row halves.
-__host__ __device__ constexpr uint32_t instr_desc(bool sparse, uint32_t afmt, uint32_t bfmt, bool b_mn_major)
+__host__ __device__ constexpr uint32_t instr_desc(bool sparse, uint32_t afmt, uint32_t bfmt, bool b_mn_major, int bn)
 {
     return (sparse ? 4u : 0u) | (1u << 4) | (afmt << 7) | (bfmt << 10) | ((b_mn_major ? 1u : 0u) << 16) |
-           (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>((2 * BM) >> 4) << 24);
+           (static_cast<uint32_t>(bn >> 3) << 17) | (static_cast<uint32_t>((2 * BM) >> 4) << 24);
 }
 
 // ------------------------------------------------------------------ kernel
@@ -221,6 +219,8 @@ struct GemmParams {
     const float *out_scale; // device scalar or null
     unsigned int *status;
     uint32_t afmt, bfmt;    // operand format codes of the instruction descriptor
+    int splits;             // split-K factor (1 = none): a work unit is (tile, K range)
+    float *partials;        // split-K: fp32 partial tiles [tile][cta][split][128][BN], summed by splitk_reduce_kernel
 #ifdef SSTE_PROBE
     int probe;              // 1: skip the loads after the first ring fill, 2: skip the MMAs
     long long *dbg;         // clock64 stamps of pair 0: [tile][0..3] = mma start, mma issued, acc full seen, epilogue done
@@ -244,29 +244,38 @@ __device__ __forceinline__ void tmem_st_32x4(uint32_t taddr, uint4 v)
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Shared-memory plan of one CTA.  A stage holds 128 bytes of K per A row and, for the sparse
-// kernels, two B sub-tiles of 128 bytes of K each (the compressed A row covers twice the K of
-// one B row); the dense kernel pairs it with one B sub-tile.
-template <bool SPARSE>
+// Shared-memory / tensor-memory plan of one CTA for a tile of 256 x BN.  A stage holds 128 bytes of K per
+// A row and, for the sparse kernels, two B sub-tiles of 128 bytes of K each (the compressed A row covers
+// twice the K of one B row); the dense kernel pairs it with one B sub-tile.  BN = 256 fills the
+// accumulator half of tensor memory with one buffer; BN <= 192 leaves room for two, so the epilogue of a
+// tile overlaps the next tile's main loop.
+template <bool SPARSE, int BN>
 struct Cfg {
     static constexpr int A_STAGE = 16384;                        // 128 rows x 128 bytes
     static constexpr int B_SUB = (BN / 2) * 128;                 // this CTA's half of one B sub-tile
     static constexpr int B_STAGE = SPARSE ? 2 * B_SUB : B_SUB;
     static constexpr int STAGE = A_STAGE + B_STAGE;
-    static constexpr int STAGES = SPARSE ? 4 : 6;
+    static constexpr int FIT = (232448 - 1024 - 512 - STAGING_BYTES) / STAGE;   // 227 KB of shared memory per CTA
+    static constexpr int STAGES = FIT > 8 ? 8 : FIT;
+    static constexpr int ACC_BUFS = (BN <= 192) ? 2 : 1;
+    static constexpr int META_COL0 = ACC_BUFS * BN;              // metadata regions follow the accumulators
     static constexpr int THREADS = SPARSE ? 320 : 192;           // + 4 metadata warps for the sparse kernels
     static constexpr int SMEM_BYTES = STAGES * STAGE + STAGING_BYTES + 1024 /* alignment slack */ + 512 /* barriers */;
+    static_assert(META_COL0 + META_REGIONS * 16 <= TMEM_COLS, "tensor memory budget");
+    static_assert(STAGES >= 3, "pipeline depth");
 };
 
 // ELT: operand element size in bytes (2 = bf16 via kind::f16, 1 = fp8 via kind::f8f6f4).
 // OUT_T: store D transposed (out[n, m]); OUT_F32: fp32 output (direct stores) instead of bf16 (TMA stores).
-template <bool SPARSE, BMajor BMAJ, int ELT, bool OUT_T, bool OUT_F32>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Cfg<SPARSE>::THREADS, 1)
+template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Cfg<SPARSE, BN>::THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const __grid_constant__ CUtensorMap map_d, const uint8_t *__restrict__ meta, const GemmParams p)
+            const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_p,
+            const uint8_t *__restrict__ meta, const GemmParams p)
 {
-    using C = Cfg<SPARSE>;
+    using C = Cfg<SPARSE, BN>;
     constexpr int NS = C::STAGES;
+    constexpr int NB = C::ACC_BUFS;
     constexpr bool F8 = (ELT == 1);
     constexpr int BK = (SPARSE ? 256 : 128) / ELT;    // logical K per stage
     constexpr int B_SUBS = SPARSE ? 2 : 1;
@@ -275,6 +284,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     constexpr int B_CHUNK_N = 128 / ELT;              // MN-major: N elements per 128-byte row
     constexpr int B_CHUNKS_HALF = (BN / 2) / B_CHUNK_N;
     constexpr uint32_t STAGE_TX = 2u * C::STAGE;      // both CTAs' operand bytes
+    constexpr int PANELS = BN / 64;                   // the epilogue works in panels of 64 columns
+    constexpr int DIRECT_PANELS = PANELS - 2;         // the last two go through registers (early release)
+    static_assert(BMAJ == BMajor::K || (BN / 2) % B_CHUNK_N == 0, "MN-major B needs whole 128-byte chunks per CTA");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -282,15 +294,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const uint32_t bars = staging + STAGING_BYTES;
     auto full_bar = [&](int s) { return bars + 8u * s; };              // used in the leader only
     auto empty_bar = [&](int s) { return bars + 8u * (NS + s); };      // one per CTA
-    const uint32_t acc_full_bar = bars + 8u * (2 * NS);                // one per CTA
-    const uint32_t acc_empty_bar = bars + 8u * (2 * NS + 1);           // leader only, 2 arrivals
-    auto meta_full_bar = [&](int r) { return bars + 8u * (2 * NS + 2 + r); };             // leader only, 8 arrivals
-    auto meta_empty_bar = [&](int r) { return bars + 8u * (2 * NS + 2 + META_REGIONS + r); };   // one per CTA
-    const uint32_t tmem_slot = bars + 8u * (2 * NS + 2 + 2 * META_REGIONS);
+    auto acc_full_bar = [&](int b) { return bars + 8u * (2 * NS + b); };           // one per CTA
+    auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * NS + 2 + b); };      // leader only, 2 arrivals
+    auto meta_full_bar = [&](int r) { return bars + 8u * (2 * NS + 4 + r); };             // leader only, 8 arrivals
+    auto meta_empty_bar = [&](int r) { return bars + 8u * (2 * NS + 4 + META_REGIONS + r); };   // one per CTA
+    constexpr int MISC = 2 * NS + 4 + 2 * META_REGIONS;
+    const uint32_t tmem_slot = bars + 8u * MISC;
     uint8_t *bars_generic = smem_raw + (bars - smem_u32(smem_raw));
-    volatile uint32_t *tmem_slot_ptr = reinterpret_cast<volatile uint32_t *>(bars_generic + 8u * (2 * NS + 2 + 2 * META_REGIONS));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_generic + 8u * (2 * NS + 3 + 2 * META_REGIONS));
+    volatile uint32_t *tmem_slot_ptr = reinterpret_cast<volatile uint32_t *>(bars_generic + 8u * MISC);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_generic + 8u * (MISC + 1));
     uint8_t *staging_generic = smem_raw + (staging - smem_u32(smem_raw));
+    static_assert(8 * (MISC + 2) <= 512, "barrier block");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -299,13 +313,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM);
     const int n_tiles = (p.N + BN - 1) / BN;
     const int num_tiles = m_tiles * n_tiles;
-    const int k_blocks = (p.K + BK - 1) / BK;         // a ragged last stage reads zero-filled K
+    const int k_blocks_total = (p.K + BK - 1) / BK;   // a ragged last stage reads zero-filled K
+    const int k_blocks = k_blocks_total / p.splits;   // stages per work unit (the host makes this exact)
+    const int num_units = num_tiles * p.splits;       // unit u = (tile u / splits, K range u % splits)
     const int k_atoms = p.K / 128;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        mbar_init(acc_full_bar, 1);
-        mbar_init(acc_empty_bar, 2);
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 2); }
         for (int r = 0; r < META_REGIONS; ++r) { mbar_init(meta_full_bar(r), 8); mbar_init(meta_empty_bar(r), 1); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -328,11 +343,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            for (int unit = pair; unit < num_units && ok; unit += num_pairs) {
+                const int tile = unit / p.splits, kb0 = (unit % p.splits) * k_blocks;
                 const int mt = tile % m_tiles, nt = tile / m_tiles;
                 const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;      // this CTA's rows of A
                 const int n0 = nt * BN + static_cast<int>(rank) * (BN / 2);    // this CTA's half of B
-                for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                for (int kb = kb0; kb < kb0 + k_blocks; ++kb, ++it) {
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1u;
                     if (PROBE_MODE(p) == 3 && it >= static_cast<uint32_t>(NS)) continue;
@@ -347,23 +363,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint32_t b_dst = a_dst + C::A_STAGE;
                     // A: 128 bytes per row = BK/2 compressed (sparse) or BK dense elements
                     tma_load_2d(a_dst, &map_a, lead_full, kb * (SPARSE ? BK / 2 : BK), m0);
+                    if (BMAJ == BMajor::K) {
 #pragma unroll
-                    for (int u = 0; u < B_SUBS; ++u) {
-                        const int k0 = kb * BK + u * SUB_K;
-                        if (BMAJ == BMajor::K) {
-                            tma_load_2d(b_dst + u * C::B_SUB, &map_b, lead_full, k0, n0);
-                        } else if (SPARSE) {
-                            // MN-major: one box per 128-byte N chunk spans the whole stage's K rows
-                            if (u == 0) {
+                        for (int u = 0; u < B_SUBS; ++u)
+                            tma_load_2d(b_dst + u * C::B_SUB, &map_b, lead_full, kb * BK + u * SUB_K, n0);
+                    } else {
+                        // MN-major: one box per 128-byte N chunk spans the whole stage's K rows
 #pragma unroll
-                                for (int c = 0; c < B_CHUNKS_HALF; ++c)
-                                    tma_load_2d(b_dst + c * (BK * 128), &map_b, lead_full, n0 + c * B_CHUNK_N, kb * BK);
-                            }
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < B_CHUNKS_HALF; ++c)
-                                tma_load_2d(b_dst + c * (BK * 128), &map_b, lead_full, n0 + c * B_CHUNK_N, kb * BK);
-                        }
+                        for (int c = 0; c < B_CHUNKS_HALF; ++c)
+                            tma_load_2d(b_dst + c * (BK * 128), &map_b, lead_full, n0 + c * B_CHUNK_N, kb * BK);
                     }
                 }
             }
@@ -371,15 +379,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (leader && lane == 0) {
-            const uint32_t idesc = instr_desc(SPARSE, p.afmt, p.bfmt, BMAJ == BMajor::MN);
+            const uint32_t idesc = instr_desc(SPARSE, p.afmt, p.bfmt, BMAJ == BMajor::MN, BN);
             uint32_t it = 0, local_tile = 0, group_it = 0;
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++local_tile) {
-                if (!mbar_wait(acc_empty_bar, (local_tile & 1u) ^ 1u, p.status, abort_flag)) { ok = false; break; }
+            for (int unit = pair; unit < num_units && ok; unit += num_pairs, ++local_tile) {
+                const uint32_t buf = local_tile % NB, use = local_tile / NB;
+                if (!mbar_wait(acc_empty_bar(buf), (use & 1u) ^ 1u, p.status, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 PROBE_STAMP(p, local_tile, 0);
-                const uint32_t d_tmem = tmem_base;
-                for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < k_blocks; ++kb, ++it) {     // stage index inside the unit's K range
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1u;
                     uint32_t meta_cols = 0;
@@ -393,7 +402,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             ok = false;
                             break;
                         }
-                        meta_cols = tmem_base + META_COL0 + 16 * region + 4 * (atom0 & 3);
+                        meta_cols = tmem_base + C::META_COL0 + 16 * region + 4 * (atom0 & 3);
                     }
                     if (!(PROBE_MODE(p) == 3 && it >= static_cast<uint32_t>(NS)) &&
                         !mbar_wait(full_bar(s), ph, p.status, abort_flag)) { ok = false; break; }
@@ -432,7 +441,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         }
                     }
                 }
-                if (ok) tc_commit_pair(acc_full_bar);
+                if (ok) tc_commit_pair(acc_full_bar(buf));
                 PROBE_STAMP(p, local_tile, 1);
             }
         }
@@ -442,22 +451,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int row = quarter * 32 + lane;           // row of this CTA's 128 x BN accumulator
         const float scale = p.out_scale ? *p.out_scale : 1.0f;
         const bool store_thread = (threadIdx.x == 64);
-        const uint32_t lead_acc_empty = map_to_cta(acc_empty_bar, 0);
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-        uint32_t local_tile = 0;
+        uint32_t local_tile = 0, panel_it = 0;
         bool ok = true;
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++local_tile) {
+        for (int unit = pair; unit < num_units && ok; unit += num_pairs, ++local_tile) {
+            const int tile = unit / p.splits, split = unit % p.splits;
             const int mt = tile % m_tiles, nt = tile / m_tiles;
             const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;
             const int n0 = nt * BN;
-            if (!mbar_wait_warp(acc_full_bar, local_tile & 1u, p.status, abort_flag)) { ok = false; break; }
+            const uint32_t buf = local_tile % NB, use = local_tile / NB;
+            const uint32_t acc_base = lane_base + buf * BN;
+            const uint32_t lead_acc_empty = map_to_cta(acc_empty_bar(buf), 0);
+            if (!mbar_wait_warp(acc_full_bar(buf), use & 1u, p.status, abort_flag)) { ok = false; break; }
             tc_fence_after();
             if (threadIdx.x == 64) PROBE_STAMP(p, local_tile, 2);
             if (OUT_F32) {
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 32) {
                     uint32_t r[32];
-                    tmem_ld_32x32(lane_base + c0, r);
+                    tmem_ld_32x32(acc_base + c0, r);
                     tmem_ld_wait();
                     const int m = m0 + row;
                     if (m < p.M && n0 + c0 < p.N) {
@@ -486,22 +498,54 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 }
                 continue;
             }
-            // bf16 output: two passes of 128 columns through a 32 KB staging buffer and TMA stores.
-            // The second half is pulled into registers first, so the accumulator is released before
-            // its conversion and stores.
-            auto stage_chunk = [&](const uint32_t (&r)[32], int c0 /* column inside the 128-column half */) {
+            if (p.splits > 1) {
+                // Split-K: the unit stores its fp32 partial tile [128][BN]; a second kernel adds the
+                // partials of a tile in split order (bit-reproducible) and writes the bf16 result.
+                // Panels of 32 fp32 columns (128-byte rows, swizzled) go out through the staging buffers and
+                // TMA stores: whole lines instead of 16-byte pieces of 32 different rows per instruction.
+                const int part_row0 = static_cast<int>(((static_cast<size_t>(tile) * 2 + rank) * p.splits + split) * BM);
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    if (store_thread) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    epilogue_barrier();
+                    const uint32_t off = (panel_it & 1u) * 16384u;
+                    uint32_t r[32];
+                    tmem_ld_32x32(acc_base + c0, r);
+                    tmem_ld_wait();
+                    uint8_t *dst = staging_generic + off + row * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4 *>(dst + ((c ^ (row & 7)) << 4)) = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+                    fence_proxy_async();
+                    epilogue_barrier();
+                    if (store_thread) {
+                        tma_store_2d(&map_p, staging + off, c0, part_row0);
+                        tma_store_commit();
+                    }
+                    ++panel_it;
+                }
+                tc_fence_before();
+                epilogue_barrier();
+                if (store_thread) {
+                    PROBE_STAMP(p, local_tile, 3);
+                    mbar_arrive_cluster(lead_acc_empty);
+                }
+                continue;
+            }
+            // bf16 output in panels of 64 columns through two 16 KB staging buffers and TMA stores.
+            // 32 accumulator columns -> bf16 -> staging buffer `sb`, columns [c0, c0 + 32) of the panel
+            auto stage_chunk = [&](const uint32_t (&r)[32], uint8_t *sb, int c0) {
                 if (OUT_T) {
-                    // staging[n][m]: 128 rows of 128 bf16; a warp writes 32 consecutive m per n
-                    uint16_t *st = reinterpret_cast<uint16_t *>(staging_generic);
+                    // staging[n][m]: 64 rows of 128 bf16; a warp writes 32 consecutive m per n
+                    uint16_t *st = reinterpret_cast<uint16_t *>(sb);
 #pragma unroll
                     for (int c = 0; c < 32; ++c)
                         st[(c0 + c) * BM + row] =
                             static_cast<uint16_t>(sste_f32_to_bf16_bits(__fmul_rn(__uint_as_float(r[c]), scale)));
                 } else {
-                    // two sub-tiles [128 rows][64 bf16] with the 128-byte swizzle of the TMA store:
-                    // 16-byte chunk index ^= row & 7
-                    uint8_t *sub = staging_generic + (c0 >> 6) * 16384 + row * 128;
-                    const int chunk0 = (c0 & 63) >> 3;
+                    // [128 rows][64 bf16] with the 128-byte swizzle of the TMA store: 16-byte chunk index ^= row & 7
+                    uint8_t *dst = sb + row * 128;
+                    const int chunk0 = c0 >> 3;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t w[4];
@@ -511,59 +555,61 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             const float hi = __fmul_rn(__uint_as_float(r[8 * c + 2 * e + 1]), scale);
                             w[e] = sste_f32_to_bf16_bits(lo) | (sste_f32_to_bf16_bits(hi) << 16);
                         }
-                        *reinterpret_cast<uint4 *>(sub + (((chunk0 + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                        *reinterpret_cast<uint4 *>(dst + (((chunk0 + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
             };
-            auto store_half = [&](int half) {
-                if (OUT_T) {
-                    tma_store_2d(&map_d, staging, m0, n0 + 128 * half);
-                } else {
-                    tma_store_2d(&map_d, staging, n0 + 128 * half, m0);
-                    tma_store_2d(&map_d, staging + 16384, n0 + 128 * half + 64, m0);
-                }
-                tma_store_commit();
+            // staging buffer of the next panel becomes writable once the store issued two panels ago has read it
+            auto acquire_staging = [&]() -> uint32_t {
+                if (store_thread) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                epilogue_barrier();
+                return (panel_it & 1u) * 16384u;
             };
-            // first half: the previous tile's store must have finished reading the staging buffer
-            if (store_thread) tma_store_wait_read();
-            epilogue_barrier();
-            {
+            auto store_panel = [&](uint32_t off, int panel) {
+                fence_proxy_async();
+                epilogue_barrier();
+                if (store_thread) {
+                    if (OUT_T) tma_store_2d(&map_d, staging + off, m0, n0 + 64 * panel);
+                    else tma_store_2d(&map_d, staging + off, n0 + 64 * panel, m0);
+                    tma_store_commit();
+                }
+                ++panel_it;
+            };
+#pragma unroll 1
+            for (int pnl = 0; pnl < DIRECT_PANELS; ++pnl) {
+                const uint32_t off = acquire_staging();
                 uint32_t ra[32], rb[32];
-                tmem_ld_32x32(lane_base + 0, ra);
-                tmem_ld_32x32(lane_base + 32, rb);
+                tmem_ld_32x32(acc_base + 64 * pnl, ra);
+                tmem_ld_32x32(acc_base + 64 * pnl + 32, rb);
                 tmem_ld_wait();
-                stage_chunk(ra, 0);
-                tmem_ld_32x32(lane_base + 64, ra);
-                stage_chunk(rb, 32);
-                tmem_ld_32x32(lane_base + 96, rb);
-                tmem_ld_wait();
-                stage_chunk(ra, 64);
-                stage_chunk(rb, 96);
+                stage_chunk(ra, staging_generic + off, 0);
+                stage_chunk(rb, staging_generic + off, 32);
+                store_panel(off, pnl);
             }
-            fence_proxy_async();
-            epilogue_barrier();
-            if (store_thread) store_half(0);
-            // second half -> registers, then the accumulator is free
+            // last two panels -> registers, then the accumulator buffer is free for the next tile
             uint32_t r0[32], r1[32], r2[32], r3[32];
-            tmem_ld_32x32(lane_base + 128, r0);
-            tmem_ld_32x32(lane_base + 160, r1);
-            tmem_ld_32x32(lane_base + 192, r2);
-            tmem_ld_32x32(lane_base + 224, r3);
+            tmem_ld_32x32(acc_base + 64 * DIRECT_PANELS, r0);
+            tmem_ld_32x32(acc_base + 64 * DIRECT_PANELS + 32, r1);
+            tmem_ld_32x32(acc_base + 64 * DIRECT_PANELS + 64, r2);
+            tmem_ld_32x32(acc_base + 64 * DIRECT_PANELS + 96, r3);
             tmem_ld_wait();
             tc_fence_before();
-            if (store_thread) tma_store_wait_read();
-            epilogue_barrier();
-            if (store_thread) {
-                PROBE_STAMP(p, local_tile, 3);
-                mbar_arrive_cluster(lead_acc_empty);
+            {
+                const uint32_t off = acquire_staging();      // includes the barrier after everyone's loads
+                if (store_thread) {
+                    PROBE_STAMP(p, local_tile, 3);
+                    mbar_arrive_cluster(lead_acc_empty);
+                }
+                stage_chunk(r0, staging_generic + off, 0);
+                stage_chunk(r1, staging_generic + off, 32);
+                store_panel(off, DIRECT_PANELS);
             }
-            stage_chunk(r0, 0);
-            stage_chunk(r1, 32);
-            stage_chunk(r2, 64);
-            stage_chunk(r3, 96);
-            fence_proxy_async();
-            epilogue_barrier();
-            if (store_thread) store_half(1);
+            {
+                const uint32_t off = acquire_staging();
+                stage_chunk(r2, staging_generic + off, 0);
+                stage_chunk(r3, staging_generic + off, 32);
+                store_panel(off, DIRECT_PANELS + 1);
+            }
         }
         if (store_thread && !OUT_F32) tma_store_wait_all();
     } else if (SPARSE) {
@@ -571,17 +617,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // HBM -> registers -> tensor memory: lane L of an atom's image is exactly the 16 bytes the
         // instruction expects in tensor-memory lane L, four 32-bit columns per atom.
         const int quarter = warp & 3;
-        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + META_COL0;
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + C::META_COL0;
         uint32_t group_it = 0;
         bool ok = true;
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        for (int unit = pair; unit < num_units && ok; unit += num_pairs) {
+            const int tile = unit / p.splits;
             const int mt = tile % m_tiles;
             const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;
             const bool rows_valid = m0 < p.M;
             const uint4 *src = reinterpret_cast<const uint4 *>(meta + static_cast<size_t>(m0 / BM) * k_atoms * 2048) +
                                quarter * 32 + lane;
-            const int atoms_padded = k_blocks * ATOMS_PER_STAGE;
-            for (int a0 = 0; a0 < atoms_padded; a0 += 4, ++group_it) {
+            const int atom_begin = (unit % p.splits) * k_blocks * ATOMS_PER_STAGE;
+            const int atom_end = atom_begin + k_blocks * ATOMS_PER_STAGE;
+            for (int a0 = atom_begin; a0 < atom_end; a0 += 4, ++group_it) {
                 const uint32_t region = group_it % META_REGIONS;
                 if (!mbar_wait_warp(meta_empty_bar(region), ((group_it / META_REGIONS) & 1u) ^ 1u, p.status, abort_flag)) {
                     ok = false;
@@ -627,19 +675,51 @@ bool make_map(const sste_ctx *ctx, CUtensorMap *map, const void *base, int elt, 
     const cuuint64_t strides[1] = {cols * static_cast<uint64_t>(elt)};
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    const CUtensorMapDataType dt = (elt == 2) ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+    const CUtensorMapDataType dt = (elt == 4)   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                   : (elt == 2) ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                                : CU_TENSOR_MAP_DATA_TYPE_UINT8;
     EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->cu_tensor_map_encode);
     return fn(map, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool SPARSE, BMajor BMAJ, int ELT, bool OUT_T, bool OUT_F32>
+int pick_splits(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn);
+
+// Split-K second pass: out[m, n] = bf16(scale * sum over splits, in split order, of the fp32 partial tiles).
+// One thread per 8 consecutive n.
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, int splits, int m_tiles,
+                     const float *__restrict__ out_scale, uint4 *__restrict__ out)
+{
+    const size_t vecs = static_cast<size_t>(M) * (N / 8);
+    const float scale = out_scale ? *out_scale : 1.0f;
+    for (size_t v = static_cast<size_t>(blockIdx.x) * 256 + threadIdx.x; v < vecs; v += static_cast<size_t>(gridDim.x) * 256) {
+        const int m = static_cast<int>(v / (N / 8)), n = static_cast<int>(v % (N / 8)) * 8;
+        const int tile = (n / bn) * m_tiles + m / (2 * BM);
+        const size_t slot = static_cast<size_t>(tile) * 2 + ((m / BM) & 1);
+        const float *src = partials + (slot * splits * BM + (m % BM)) * bn + (n % bn);
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int s = 0; s < splits; ++s) {
+            const float4 a = __ldcg(reinterpret_cast<const float4 *>(src + static_cast<size_t>(s) * BM * bn));
+            const float4 b = __ldcg(reinterpret_cast<const float4 *>(src + static_cast<size_t>(s) * BM * bn) + 1);
+            acc[0] = __fadd_rn(acc[0], a.x); acc[1] = __fadd_rn(acc[1], a.y); acc[2] = __fadd_rn(acc[2], a.z); acc[3] = __fadd_rn(acc[3], a.w);
+            acc[4] = __fadd_rn(acc[4], b.x); acc[5] = __fadd_rn(acc[5], b.y); acc[6] = __fadd_rn(acc[6], b.z); acc[7] = __fadd_rn(acc[7], b.w);
+        }
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            w[e] = sste_f32_to_bf16_bits(__fmul_rn(acc[2 * e], scale)) | (sste_f32_to_bf16_bits(__fmul_rn(acc[2 * e + 1], scale)) << 16);
+        out[v] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32>
 sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void *meta, const GemmParams &p,
                    cudaStream_t stream)
 {
-    using C = Cfg<SPARSE>;
+    using C = Cfg<SPARSE, BN>;
     constexpr int BK = (SPARSE ? 256 : 128) / ELT;
-    CUtensorMap map_a, map_b, map_d;
+    CUtensorMap map_a, map_b, map_d, map_p;
     bool ok;
     if (SPARSE)   // compressed values [M, K/2]: 128 bytes per row per stage
         ok = make_map(ctx, &map_a, A, ELT, p.M, p.K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -651,13 +731,13 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         ok = ok && make_map(ctx, &map_b, B, ELT, p.K, p.N, 128 / ELT, BK, CU_TENSOR_MAP_SWIZZLE_128B);
     if (OUT_F32) {
         map_d = map_a;       // unused: the fp32 epilogue stores directly
-    } else if (OUT_T) {      // out[N, M] bf16: box = 128 m x 128 n
-        ok = ok && make_map(ctx, &map_d, p.D, 2, p.N, p.M, BM, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
-    } else {                 // out[M, N] bf16: boxes of 64 n x 128 m, 128-byte swizzle
+    } else if (OUT_T) {      // out[N, M] bf16: panels of 128 m x 64 n
+        ok = ok && make_map(ctx, &map_d, p.D, 2, p.N, p.M, BM, 64, CU_TENSOR_MAP_SWIZZLE_NONE);
+    } else {                 // out[M, N] bf16: panels of 64 n x 128 m, 128-byte swizzle
         ok = ok && make_map(ctx, &map_d, p.D, 2, p.M, p.N, 64, BM, CU_TENSOR_MAP_SWIZZLE_128B);
     }
     if (!ok) return SSTE_ERR_CUDA;
-    auto kern = gemm_kernel<SPARSE, BMAJ, ELT, OUT_T, OUT_F32>;
+    auto kern = gemm_kernel<SPARSE, BMAJ, ELT, BN, OUT_T, OUT_F32>;
     static bool attr_set = false;   // per instantiation
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
@@ -665,15 +745,62 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         attr_set = true;
     }
     const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM), n_tiles = (p.N + BN - 1) / BN;
-    int pairs = m_tiles * n_tiles;
-    if (pairs > ctx->sm_count / 2) pairs = ctx->sm_count / 2;
     GemmParams pp = p;
+    pp.splits = (OUT_F32 || OUT_T) ? 1 : pick_splits(ctx, m_tiles * n_tiles, (p.K + BK - 1) / BK, SPARSE ? 4 / (BK / 128) : 1, BN);
+    pp.partials = ctx->splitk_partials;
+    int pairs = m_tiles * n_tiles * pp.splits;
+    if (pairs > ctx->sm_count / 2) pairs = ctx->sm_count / 2;
 #ifdef SSTE_PROBE
     pp.probe = g_probe_mode;
     pp.dbg = g_probe_dbg;
 #endif
-    kern<<<2 * pairs, C::THREADS, C::SMEM_BYTES, stream>>>(map_a, map_b, map_d, static_cast<const uint8_t *>(meta), pp);
+    map_p = map_a;   // unused without split-K
+    if (pp.splits > 1 &&
+        !make_map(ctx, &map_p, pp.partials, 4, static_cast<uint64_t>(m_tiles) * n_tiles * 2 * pp.splits * BM, BN, 32, BM,
+                  CU_TENSOR_MAP_SWIZZLE_128B))
+        return SSTE_ERR_CUDA;
+    kern<<<2 * pairs, C::THREADS, C::SMEM_BYTES, stream>>>(map_a, map_b, map_d, map_p, static_cast<const uint8_t *>(meta), pp);
+    if (pp.splits > 1) {
+        const size_t vecs = static_cast<size_t>(p.M) * (p.N / 8);
+        size_t blocks = (vecs + 255) / 256;
+        if (blocks > static_cast<size_t>(ctx->sm_count) * 16) blocks = static_cast<size_t>(ctx->sm_count) * 16;
+        splitk_reduce_kernel<<<static_cast<unsigned int>(blocks), 256, 0, stream>>>(
+            pp.partials, p.M, p.N, BN, pp.splits, m_tiles, p.out_scale, static_cast<uint4 *>(p.D));
+    }
     return cudaGetLastError() == cudaSuccess ? SSTE_OK : SSTE_ERR_CUDA;
+}
+
+int g_force_splits = 0;   // test hook: 0 = automatic split-K factor
+
+// Split-K factor for products with few output tiles and a long reduction (the weight gradient of a
+// GPT-2-sized layer has 36 tiles for 74 CTA pairs).  A work unit is (tile, K range); time goes like
+// waves(units) * K / splits, plus a few percent per extra split for the fp32 partial round trip.
+// `align` = stages per metadata group (the K ranges must start on a group boundary).
+int pick_splits(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn)
+{
+    if (!ctx->splitk_partials) return 1;
+    const int pairs = ctx->sm_count / 2;
+    int best = 1;
+    double best_cost = 0.0;
+    for (int s = 1; s <= 4; ++s) {
+        if (k_blocks % (s * align) != 0 || k_blocks / s < 8) continue;
+        if (static_cast<size_t>(tiles) * 2 * s * BM * bn * sizeof(float) > ctx->splitk_partial_bytes) continue;
+        if (g_force_splits == s) return s;
+        if (2 * tiles > pairs) continue;   // splitting pays only while less than half of the pairs have a tile
+        const int waves = (tiles * s + pairs - 1) / pairs;
+        const double cost = static_cast<double>(waves) / s + 0.06 * (s - 1);
+        if (s == 1 || cost < best_cost - 1e-9) { best = s; best_cost = cost; }
+    }
+    return best;
+}
+
+// Tile width, from timings on B200 over the GPT-2- and 7B-shaped layers: 256 columns is the fastest
+// almost everywhere (least L2 -> shared-memory traffic per flop); only the forward with a short
+// reduction (K <= 1024) gains from 192 columns, where the second accumulator buffer hides an
+// epilogue that is as long as the main loop.
+int pick_bn(bool b_k_major, int K)
+{
+    return (b_k_major && K <= 1024) ? 192 : 256;
 }
 
 bool fmt_code(sste_dtype dt, int *elt, uint32_t *code)
@@ -686,19 +813,47 @@ bool fmt_code(sste_dtype dt, int *elt, uint32_t *code)
     }
 }
 
-// dispatch on output dtype
+int g_force_bn = 0;   // test hook: 0 = automatic tile width
+
+// Dispatch on tile width and output dtype.  fp32 output (a test / debug path) always uses 256-wide tiles.
 template <bool SPARSE, BMajor BMAJ, int ELT, bool OUT_T>
 sste_status launch_out(const sste_ctx *ctx, const void *A, const void *B, const void *meta, const GemmParams &p,
                        sste_dtype odt, cudaStream_t s)
 {
-    if (odt == SSTE_F32) return launch<SPARSE, BMAJ, ELT, OUT_T, true>(ctx, A, B, meta, p, s);
-    if (odt == SSTE_BF16) return launch<SPARSE, BMAJ, ELT, OUT_T, false>(ctx, A, B, meta, p, s);
-    return SSTE_ERR_DTYPE;
+    if (odt == SSTE_F32) return launch<SPARSE, BMAJ, ELT, 256, OUT_T, true>(ctx, A, B, meta, p, s);
+    if (odt != SSTE_BF16) return SSTE_ERR_DTYPE;
+    constexpr bool MN = (BMAJ == BMajor::MN);
+    int cands[3], n = 0;
+    cands[n++] = 256;
+    if (!(MN && ELT == 1)) cands[n++] = 128;   // MN-major B: each CTA needs whole 128-byte chunks of N
+    if (!MN) cands[n++] = 192;
+    int bn = pick_bn(!MN, p.K);
+    for (int i = 0; i < n; ++i)
+        if (cands[i] == g_force_bn) bn = g_force_bn;
+    if constexpr (!MN) {
+        if (bn == 192) return launch<SPARSE, BMAJ, ELT, 192, OUT_T, false>(ctx, A, B, meta, p, s);
+    }
+    if constexpr (!(MN && ELT == 1)) {
+        if (bn == 128) return launch<SPARSE, BMAJ, ELT, 128, OUT_T, false>(ctx, A, B, meta, p, s);
+    }
+    return launch<SPARSE, BMAJ, ELT, 256, OUT_T, false>(ctx, A, B, meta, p, s);
 }
 
 }  // namespace
 
 sste_status sste_gemm_launch_check(const sste_ctx *) { return SSTE_OK; }
+extern "C" sste_status sste_debug_force_splits(int splits)
+{
+    if (splits < 0 || splits > 4) return SSTE_ERR_INVALID_ARG;
+    g_force_splits = splits;
+    return SSTE_OK;
+}
+extern "C" sste_status sste_debug_force_tile_width(int bn)
+{
+    if (bn != 0 && bn != 128 && bn != 192 && bn != 256) return SSTE_ERR_INVALID_ARG;
+    g_force_bn = bn;
+    return SSTE_OK;
+}
 #ifdef SSTE_PROBE
 extern "C" void sste_probe_set_mode(int mode) { g_probe_mode = mode; }
 extern "C" void sste_probe_set_dbg(long long *dbg) { g_probe_dbg = dbg; }

@@ -97,8 +97,9 @@ def test_mvue_e5m2(ctx, T, O):
     assert np.array_equal(canonical_meta(ctx, m16, O, T, B.BF16), ogm)
 
 
+@pytest.mark.parametrize("tile_width", [0, 128, 192, 256])
 @pytest.mark.parametrize("O,I,T", [(256, 256, 512), (384, 640, 1152), (128, 384, 128)])
-def test_fp8_products(ctx, O, I, T):
+def test_fp8_products(ctx, O, I, T, tile_width):
     """Each product against the fp64 product of the decoded FP8 operands, times 1/(scale_a * scale_b)."""
     from paper_2409_09099_b200 import binding as B
     W = synth.gaussian_bf16(O + 11, (O, I), 0.02)
@@ -117,6 +118,7 @@ def test_fp8_products(ctx, O, I, T):
     gvals, gmeta = ctx.alloc_compressed(O, T, B.E5M2)
     dYq = torch.empty((T, O), dtype=torch.float8_e5m2, device=DEV)
     ctx.mvue_sparsify(dbf16(dY), 5, 0, 0, gvals, gmeta, dense_q_out=dYq, gscale_dev=_f32(sg))
+    ctx.debug_force_tile_width(tile_width)
     inv_xw = np.float32(np.float32(1) / sx) * np.float32(np.float32(1) / sw)
     inv_gx = np.float32(np.float32(1) / sg) * np.float32(np.float32(1) / sx)
     inv_gw = np.float32(np.float32(1) / sg) * np.float32(np.float32(1) / sw)
@@ -136,6 +138,7 @@ def test_fp8_products(ctx, O, I, T):
         assert rel_fro(Y.float().cpu().numpy(), Y_ref) <= tol
         assert rel_fro(dW.float().cpu().numpy(), dW_ref) <= tol
         assert rel_fro(dX.float().cpu().numpy(), dX_ref) <= tol
+    ctx.debug_force_tile_width(0)
     # reported, not gated: distance to the unquantised bf16 path
     Y16 = orc.linear_fwd(X, orc.BF16, *orc.project_compress(W, beta32)[:2], orc.BF16)
     assert rel_fro(Y_ref, Y16) < 0.1

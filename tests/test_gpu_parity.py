@@ -107,10 +107,20 @@ def test_mvue_sparsify(ctx, O, I, T):
     assert np.array_equal(bits16(gvals2), orc.mvue(dY, seed, tid, step + 1)[0])
 
 
-@pytest.mark.parametrize("O,I,T", SHAPES)
+@pytest.fixture(params=[0, 128, 192, 256])
+def tile_width(request, ctx):
+    """Every tile-width variant of the product kernels (0 = the library's own choice)."""
+    ctx.debug_force_tile_width(request.param)
+    yield request.param
+    ctx.debug_force_tile_width(0)
+
+
+@pytest.mark.parametrize("O,I,T", SHAPES + [(768, 512, 1024)])
 @pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
-def test_three_products(ctx, O, I, T, out_dtype):
+def test_three_products(ctx, O, I, T, out_dtype, tile_width):
     from paper_2409_09099_b200 import binding as B
+    if out_dtype == torch.float32 and tile_width not in (0, 256):
+        pytest.skip("fp32 output always uses 256-wide tiles")
     W, X, dY = _adversarial_weight(O, O, I), synth.gaussian_bf16(O + 1, (T, I), 1.0), synth.gaussian_bf16(O + 2, (T, O), 1e-2)
     Wd, Xd, dYd = dbf16(W), dbf16(X), dbf16(dY)
     beta_dev = torch.zeros(1, dtype=torch.float32, device=DEV)
@@ -145,6 +155,66 @@ def test_three_products(ctx, O, I, T, out_dtype):
     Y2 = torch.empty_like(Y)
     ctx.linear_fwd(Xd, vals, meta, Y2, out_scale_dev=sc)
     assert torch.equal(Y2.float(), Y.float() * 0.25)
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 4])
+@pytest.mark.parametrize("O,I,T", [(256, 3072, 3072), (2048, 256, 512)])
+def test_split_k_products(ctx, O, I, T, splits):
+    """Split-K (fp32 partial tiles in the workspace, summed in split order) gives the same products,
+    bit for bit from run to run, for every split factor the shape allows."""
+    from paper_2409_09099_b200 import binding as B
+    W, X, dY = synth.gaussian_bf16(O + 5, (O, I), 0.02), synth.gaussian_bf16(O + 6, (T, I), 1.0), synth.gaussian_bf16(O + 7, (T, O), 1e-2)
+    Wd, Xd, dYd = dbf16(W), dbf16(X), dbf16(dY)
+    beta_dev = torch.zeros(1, dtype=torch.float32, device=DEV)
+    ctx.beta_init(Wd, beta_dev)
+    vals, meta = ctx.alloc_compressed(O, I)
+    dense = torch.empty((O, I), dtype=torch.bfloat16, device=DEV)
+    ctx.project_compress(Wd, beta_dev, vals, meta, dense)
+    gvals, gmeta = ctx.alloc_compressed(O, T)
+    ctx.mvue_sparsify(dYd, 7, 1, 0, gvals, gmeta)
+    outs = []
+    ctx.debug_force_splits(splits)
+    try:
+        for rep in range(2):
+            Y = torch.empty((T, O), dtype=torch.bfloat16, device=DEV)
+            dW = torch.empty((O, I), dtype=torch.bfloat16, device=DEV)
+            dX = torch.empty((T, I), dtype=torch.bfloat16, device=DEV)
+            ctx.linear_fwd(Xd, vals, meta, Y)
+            ctx.linear_bwd_weight(gvals, gmeta, Xd, dW)
+            ctx.linear_bwd_input(dYd, dense, dX)
+            torch.cuda.synchronize()
+            outs.append((Y, dW, dX))
+    finally:
+        ctx.debug_force_splits(0)
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    Y, dW, dX = outs[0]
+    Y_ref = orc.linear_fwd(X, orc.BF16, bits16(vals), canonical_meta(ctx, meta, O, I, B.BF16), orc.BF16)
+    dW_ref = orc.linear_bwd_weight(bits16(gvals), canonical_meta(ctx, gmeta, O, T, B.BF16), orc.BF16, X, orc.BF16)
+    dX_ref = orc.linear_bwd_input(dY, orc.BF16, bits16(dense), orc.BF16)
+    assert rel_fro(Y.float().cpu().numpy(), Y_ref) <= BF16_GEMM_TOL
+    assert rel_fro(dW.float().cpu().numpy(), dW_ref) <= BF16_GEMM_TOL
+    assert rel_fro(dX.float().cpu().numpy(), dX_ref) <= BF16_GEMM_TOL
+    assert ctx.poll_device_status() == 0
+
+
+def test_minimal_workspace_never_splits():
+    """A context created with the minimal workspace has no room for partial tiles and still computes."""
+    from paper_2409_09099_b200 import binding as B
+    c = B.Context(0, minimal_workspace=True)
+    O, I, T = 256, 256, 4096
+    X = synth.gaussian_bf16(1, (T, I), 1.0)
+    dY = synth.gaussian_bf16(2, (T, O), 1e-2)
+    gvals, gmeta = c.alloc_compressed(O, T)
+    c.mvue_sparsify(dbf16(dY), 1, 0, 0, gvals, gmeta)
+    dW = torch.empty((O, I), dtype=torch.bfloat16, device=DEV)
+    c.debug_force_splits(4)
+    c.linear_bwd_weight(gvals, gmeta, dbf16(X), dW)
+    c.debug_force_splits(0)
+    ref = orc.linear_bwd_weight(bits16(gvals), canonical_meta(c, gmeta, O, T, B.BF16), orc.BF16, X, orc.BF16)
+    assert rel_fro(dW.float().cpu().numpy(), ref) <= BF16_GEMM_TOL
+    assert c.poll_device_status() == 0
+    c.close()
 
 
 def test_forward_of_already_sparse_weight_is_the_dense_product(ctx):
