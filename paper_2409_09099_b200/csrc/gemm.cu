@@ -219,7 +219,8 @@ struct GemmParams {
     const float *out_scale; // device scalar or null
     unsigned int *status;
     uint32_t afmt, bfmt;    // operand format codes of the instruction descriptor
-    int splits;             // split-K factor (1 = none): a work unit is (tile, K range)
+    int splits;             // split-K factor of the tiles from `split_from` on (1 = none)
+    int split_from;         // first split tile: tiles below it are computed whole
     float *partials;        // split-K: fp32 partial tiles [tile][cta][split][128][BN], summed by splitk_reduce_kernel
 #ifdef SSTE_PROBE
     int probe;              // 1: skip the loads after the first ring fill, 2: skip the MMAs
@@ -314,8 +315,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int n_tiles = (p.N + BN - 1) / BN;
     const int num_tiles = m_tiles * n_tiles;
     const int k_blocks_total = (p.K + BK - 1) / BK;   // a ragged last stage reads zero-filled K
-    const int k_blocks = k_blocks_total / p.splits;   // stages per work unit (the host makes this exact)
-    const int num_units = num_tiles * p.splits;       // unit u = (tile u / splits, K range u % splits)
+    // Work units: tiles [0, split_from) are whole; every later tile is cut into `splits` K ranges (the
+    // host makes the division exact).  Whole tiles fill complete waves, the split ones spread the
+    // last, partial wave over all pairs.
+    const int num_units = p.split_from + (num_tiles - p.split_from) * p.splits;
+    struct Unit { int tile, split, k_blocks; };
+    auto decode = [&](int unit) {
+        Unit u;
+        if (unit < p.split_from) { u.tile = unit; u.split = 0; u.k_blocks = k_blocks_total; }
+        else {
+            const int v = unit - p.split_from;
+            u.tile = p.split_from + v / p.splits;
+            u.split = v % p.splits;
+            u.k_blocks = k_blocks_total / p.splits;
+        }
+        return u;
+    };
     const int k_atoms = p.K / 128;
 
     if (threadIdx.x == 0) {
@@ -344,7 +359,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             uint32_t it = 0;
             bool ok = true;
             for (int unit = pair; unit < num_units && ok; unit += num_pairs) {
-                const int tile = unit / p.splits, kb0 = (unit % p.splits) * k_blocks;
+                const Unit u = decode(unit);
+                const int tile = u.tile, k_blocks = u.k_blocks, kb0 = u.split * u.k_blocks;
                 const int mt = tile % m_tiles, nt = tile / m_tiles;
                 const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;      // this CTA's rows of A
                 const int n0 = nt * BN + static_cast<int>(rank) * (BN / 2);    // this CTA's half of B
@@ -383,6 +399,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             uint32_t it = 0, local_tile = 0, group_it = 0;
             bool ok = true;
             for (int unit = pair; unit < num_units && ok; unit += num_pairs, ++local_tile) {
+                const int k_blocks = decode(unit).k_blocks;
                 const uint32_t buf = local_tile % NB, use = local_tile / NB;
                 if (!mbar_wait(acc_empty_bar(buf), (use & 1u) ^ 1u, p.status, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -455,7 +472,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint32_t local_tile = 0, panel_it = 0;
         bool ok = true;
         for (int unit = pair; unit < num_units && ok; unit += num_pairs, ++local_tile) {
-            const int tile = unit / p.splits, split = unit % p.splits;
+            const Unit u = decode(unit);
+            const int tile = u.tile, split = u.split;
             const int mt = tile % m_tiles, nt = tile / m_tiles;
             const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;
             const int n0 = nt * BN;
@@ -498,12 +516,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 }
                 continue;
             }
-            if (p.splits > 1) {
+            if (unit >= p.split_from && p.splits > 1) {
                 // Split-K: the unit stores its fp32 partial tile [128][BN]; a second kernel adds the
                 // partials of a tile in split order (bit-reproducible) and writes the bf16 result.
                 // Panels of 32 fp32 columns (128-byte rows, swizzled) go out through the staging buffers and
                 // TMA stores: whole lines instead of 16-byte pieces of 32 different rows per instruction.
-                const int part_row0 = static_cast<int>(((static_cast<size_t>(tile) * 2 + rank) * p.splits + split) * BM);
+                const int part_row0 =
+                    static_cast<int>(((static_cast<size_t>(tile - p.split_from) * 2 + rank) * p.splits + split) * BM);
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 32) {
                     if (store_thread) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
@@ -621,13 +640,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint32_t group_it = 0;
         bool ok = true;
         for (int unit = pair; unit < num_units && ok; unit += num_pairs) {
-            const int tile = unit / p.splits;
+            const Unit u = decode(unit);
+            const int tile = u.tile, k_blocks = u.k_blocks;
             const int mt = tile % m_tiles;
             const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;
             const bool rows_valid = m0 < p.M;
             const uint4 *src = reinterpret_cast<const uint4 *>(meta + static_cast<size_t>(m0 / BM) * k_atoms * 2048) +
                                quarter * 32 + lane;
-            const int atom_begin = (unit % p.splits) * k_blocks * ATOMS_PER_STAGE;
+            const int atom_begin = u.split * k_blocks * ATOMS_PER_STAGE;
             const int atom_end = atom_begin + k_blocks * ATOMS_PER_STAGE;
             for (int a0 = atom_begin; a0 < atom_end; a0 += 4, ++group_it) {
                 const uint32_t region = group_it % META_REGIONS;
@@ -683,21 +703,24 @@ bool make_map(const sste_ctx *ctx, CUtensorMap *map, const void *base, int elt, 
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int pick_splits(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn);
-
-// Split-K second pass: out[m, n] = bf16(scale * sum over splits, in split order, of the fp32 partial tiles).
-// One thread per 8 consecutive n.
+// Split-K second pass over the split tiles: out[m, n] = bf16(scale * sum over splits, in split order, of
+// the fp32 partial tiles [split tile][cta][split][128][bn]).  One thread per 8 consecutive n.
 __global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, int splits, int m_tiles,
-                     const float *__restrict__ out_scale, uint4 *__restrict__ out)
+splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, int splits, int m_tiles, int split_from,
+                     int n_split_tiles, const float *__restrict__ out_scale, uint4 *__restrict__ out)
 {
-    const size_t vecs = static_cast<size_t>(M) * (N / 8);
+    const int vec_per_row = bn / 8;
+    const size_t vecs = static_cast<size_t>(n_split_tiles) * 2 * BM * vec_per_row;
     const float scale = out_scale ? *out_scale : 1.0f;
     for (size_t v = static_cast<size_t>(blockIdx.x) * 256 + threadIdx.x; v < vecs; v += static_cast<size_t>(gridDim.x) * 256) {
-        const int m = static_cast<int>(v / (N / 8)), n = static_cast<int>(v % (N / 8)) * 8;
-        const int tile = (n / bn) * m_tiles + m / (2 * BM);
-        const size_t slot = static_cast<size_t>(tile) * 2 + ((m / BM) & 1);
-        const float *src = partials + (slot * splits * BM + (m % BM)) * bn + (n % bn);
+        const int col = static_cast<int>(v % vec_per_row) * 8;
+        const int row = static_cast<int>((v / vec_per_row) % BM);
+        const size_t slot = v / (static_cast<size_t>(vec_per_row) * BM);        // (split tile, cta)
+        const int tile = split_from + static_cast<int>(slot >> 1);
+        const int m = (tile % m_tiles) * 2 * BM + static_cast<int>(slot & 1) * BM + row;
+        const int n = (tile / m_tiles) * bn + col;
+        if (m >= M || n >= N) continue;
+        const float *src = partials + (slot * splits * BM + row) * bn + col;
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int s = 0; s < splits; ++s) {
             const float4 a = __ldcg(reinterpret_cast<const float4 *>(src + static_cast<size_t>(s) * BM * bn));
@@ -709,9 +732,12 @@ splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, i
 #pragma unroll
         for (int e = 0; e < 4; ++e)
             w[e] = sste_f32_to_bf16_bits(__fmul_rn(acc[2 * e], scale)) | (sste_f32_to_bf16_bits(__fmul_rn(acc[2 * e + 1], scale)) << 16);
-        out[v] = make_uint4(w[0], w[1], w[2], w[3]);
+        out[(static_cast<size_t>(m) * N + n) / 8] = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
+
+struct SplitPlan { int splits, split_from; };
+SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn);
 
 template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32>
 sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void *meta, const GemmParams &p,
@@ -746,9 +772,14 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
     }
     const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM), n_tiles = (p.N + BN - 1) / BN;
     GemmParams pp = p;
-    pp.splits = (OUT_F32 || OUT_T) ? 1 : pick_splits(ctx, m_tiles * n_tiles, (p.K + BK - 1) / BK, SPARSE ? 4 / (BK / 128) : 1, BN);
+    const int tiles = m_tiles * n_tiles;
+    SplitPlan plan{1, tiles};
+    if (!OUT_F32 && !OUT_T) plan = pick_split_plan(ctx, tiles, (p.K + BK - 1) / BK, SPARSE ? 4 / (BK / 128) : 1, BN);
+    pp.splits = plan.splits;
+    pp.split_from = plan.split_from;
     pp.partials = ctx->splitk_partials;
-    int pairs = m_tiles * n_tiles * pp.splits;
+    const int n_split_tiles = tiles - pp.split_from;
+    int pairs = pp.split_from + n_split_tiles * pp.splits;
     if (pairs > ctx->sm_count / 2) pairs = ctx->sm_count / 2;
 #ifdef SSTE_PROBE
     pp.probe = g_probe_mode;
@@ -756,42 +787,47 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
 #endif
     map_p = map_a;   // unused without split-K
     if (pp.splits > 1 &&
-        !make_map(ctx, &map_p, pp.partials, 4, static_cast<uint64_t>(m_tiles) * n_tiles * 2 * pp.splits * BM, BN, 32, BM,
+        !make_map(ctx, &map_p, pp.partials, 4, static_cast<uint64_t>(n_split_tiles) * 2 * pp.splits * BM, BN, 32, BM,
                   CU_TENSOR_MAP_SWIZZLE_128B))
         return SSTE_ERR_CUDA;
     kern<<<2 * pairs, C::THREADS, C::SMEM_BYTES, stream>>>(map_a, map_b, map_d, map_p, static_cast<const uint8_t *>(meta), pp);
     if (pp.splits > 1) {
-        const size_t vecs = static_cast<size_t>(p.M) * (p.N / 8);
+        const size_t vecs = static_cast<size_t>(n_split_tiles) * 2 * BM * (BN / 8);
         size_t blocks = (vecs + 255) / 256;
         if (blocks > static_cast<size_t>(ctx->sm_count) * 16) blocks = static_cast<size_t>(ctx->sm_count) * 16;
         splitk_reduce_kernel<<<static_cast<unsigned int>(blocks), 256, 0, stream>>>(
-            pp.partials, p.M, p.N, BN, pp.splits, m_tiles, p.out_scale, static_cast<uint4 *>(p.D));
+            pp.partials, p.M, p.N, BN, pp.splits, m_tiles, pp.split_from, n_split_tiles, p.out_scale,
+            static_cast<uint4 *>(p.D));
     }
     return cudaGetLastError() == cudaSuccess ? SSTE_OK : SSTE_ERR_CUDA;
 }
 
 int g_force_splits = 0;   // test hook: 0 = automatic split-K factor
 
-// Split-K factor for products with few output tiles and a long reduction (the weight gradient of a
-// GPT-2-sized layer has 36 tiles for 74 CTA pairs).  A work unit is (tile, K range); time goes like
-// waves(units) * K / splits, plus a few percent per extra split for the fp32 partial round trip.
-// `align` = stages per metadata group (the K ranges must start on a group boundary).
-int pick_splits(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn)
+// Split-K plan.  Tiles that fill complete waves of CTA pairs are computed whole; the tiles of the last,
+// partial wave (all of them when there are fewer tiles than pairs, as for the weight gradient of a
+// GPT-2-sized layer: 36 tiles, 74 pairs) are cut into `splits` K ranges so that the wave takes 1/splits
+// of a tile time.  `align` = stages per metadata group (K ranges must start on a group boundary).
+SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn)
 {
-    if (!ctx->splitk_partials) return 1;
+    SplitPlan none{1, tiles};
+    if (!ctx->splitk_partials) return none;
     const int pairs = ctx->sm_count / 2;
+    const int whole = (tiles / pairs) * pairs;
+    const int tail = tiles - whole;
+    if (tail == 0) return none;
     int best = 1;
-    double best_cost = 0.0;
-    for (int s = 1; s <= 4; ++s) {
+    double best_cost = 1.0;            // time of the last wave in units of one whole tile
+    for (int s = 2; s <= 4; ++s) {
         if (k_blocks % (s * align) != 0 || k_blocks / s < 8) continue;
-        if (static_cast<size_t>(tiles) * 2 * s * BM * bn * sizeof(float) > ctx->splitk_partial_bytes) continue;
-        if (g_force_splits == s) return s;
-        if (2 * tiles > pairs) continue;   // splitting pays only while less than half of the pairs have a tile
-        const int waves = (tiles * s + pairs - 1) / pairs;
-        const double cost = static_cast<double>(waves) / s + 0.06 * (s - 1);
-        if (s == 1 || cost < best_cost - 1e-9) { best = s; best_cost = cost; }
+        if (static_cast<size_t>(tail) * 2 * s * BM * bn * sizeof(float) > ctx->splitk_partial_bytes) continue;
+        if (g_force_splits == s) return SplitPlan{s, whole};
+        const int waves = (tail * s + pairs - 1) / pairs;
+        const double cost = static_cast<double>(waves) / s + 0.08 * s;   // + partial tiles' round trip
+        if (cost < best_cost - 1e-9) { best = s; best_cost = cost; }
     }
-    return best;
+    if (g_force_splits == 1 || best == 1) return none;
+    return SplitPlan{best, whole};
 }
 
 // Tile width, from timings on B200 over the GPT-2- and 7B-shaped layers: 256 columns is the fastest
