@@ -151,7 +151,7 @@ def run_reference(args):
 def workload_config(cfg_id, cfg, n_gpus):
     return {"workload": f"BASELINE config {cfg_id}: " + ", ".join(f"{L.name} W[{L.O},{L.I}] x {L.T} tokens" for L in cfg["layers"]),
             "precision": "fp8 (e4m3 fwd / e5m2 bwd)" if cfg["fp8"] else "bf16",
-            "tokens_per_gpu": cfg["layers"][0].T, "parallelism": f"dp{n_gpus} (token shards, no data-path collective)",
+            "tokens_per_gpu": cfg["layers"][0].T, "parallelism": f"dp{n_gpus} (token shards; grad_W all-reduced over NCCL when n_gpus > 1)",
             "l2": "flushed between timed steps (512 MiB write)", "launch": "one CUDA-graph replay per step"}
 
 
@@ -162,7 +162,7 @@ def run_gpu(args):
     import torch
     import torch.distributed as dist
 
-    from paper_2409_09099_b200 import binding as B, synth
+    from paper_2409_09099_b200 import binding as B, dp, synth
     from paper_2409_09099_b200.layer import SsteLinear
 
     rank = int(os.environ.get("RANK", "0"))
@@ -181,7 +181,9 @@ def run_gpu(args):
     def to_dev(a):
         return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
 
-    # weak scaling: every rank holds the full weights and its own batch of tokens (seeded per rank)
+    # weak scaling: every rank holds the full weights and its own batch of tokens (seeded per rank); the
+    # global batch is world x T tokens and a rank's MVUE counter starts at its first token
+    token_offset = rank * cfg["layers"][0].T
     layers, host = [], []
     flops_step = 0.0
     for li, L in enumerate(cfg["layers"]):
@@ -206,20 +208,25 @@ def run_gpu(args):
                 e = torch.cuda.Event(enable_timing=True)
                 e.record(stream)
                 events.append(e)
+        handles = []
         for lin, X, dY in layers:
             mark(); lin.prune()
             mark(); lin.forward(X)
             mark()
             if fp8:
-                lin.backward(dY, step_idx)
+                lin.backward(dY, step_idx, token_offset=token_offset)
                 mark(); mark(); mark()
             else:
                 c = lin.ctx
-                c.mvue_sparsify(dY, lin.seed, lin.tensor_id, step_idx, lin.gvals, lin.gmeta)
+                c.mvue_sparsify(dY, lin.seed, lin.tensor_id, step_idx, lin.gvals, lin.gmeta, token_offset=token_offset)
                 mark(); c.linear_bwd_weight(lin.gvals, lin.gmeta, lin.X, lin.dW)
                 mark(); c.linear_bwd_input(dY, lin.w_dense, lin.dX)
                 mark()
                 lin.launches += 3
+            # data parallel: the per-rank partial grad_W is summed over ranks (the path's one exchange step)
+            handles += dp.allreduce_grad_w([lin.dW])
+        for h in handles:
+            h.wait()
 
     def barrier():
         if world > 1:
@@ -233,7 +240,7 @@ def run_gpu(args):
     # The timed step is one CUDA-graph replay of all launches of the step (no host work between kernels);
     # the MVUE step counter is frozen in the graph, which does not change the work done.
     graph = None
-    if not args.no_graph:
+    if not args.no_graph and world == 1:      # collectives are launched eagerly
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
             step(args.warmup)

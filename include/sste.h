@@ -131,15 +131,18 @@ sste_status sste_linear_fwd(sste_ctx *ctx, const void *X, int T, const void *val
  * Sec. 5.1: minimum-variance unbiased 2:4 sparsification of grad_Z^T (the paper applies MVUE to
  * the output gradient only).  Groups are 4 consecutive tokens of one output column.  Inclusion
  * probabilities p_i = min(1, c|a_i|), sum 2; kept values a_i / p_i; joint law = systematic
- * sampling with one uniform per group.  Group (column j, token group tg) has index
- * g = tg*O + j; Philox4x32-10 with counter (lo32(g>>2), hi32(g>>2), tensor_id, step) and key
+ * sampling with one uniform per group.  Group (column j, token group tg) has the GLOBAL index
+ * g = (token_offset/4 + tg)*O + j, where token_offset is the number of tokens that precede this
+ * call's dY in the whole batch (0 on one GPU; a data-parallel rank passes the start of its token
+ * shard, a multiple of 4, so that the draws do not depend on how the batch is sharded).
+ * Philox4x32-10 with counter (lo32(g>>2), hi32(g>>2), tensor_id, step) and key
  * (lo32(seed), hi32(seed)); the group uses output word g&3, u = (word >> 8) * 2^-24.
  * dY: bf16 [T, O].  odt: SSTE_BF16, or SSTE_E5M2 with values fl32(v * gscale) (gscale_dev
  * non-NULL).  Outputs: the compressed operand of the TRANSPOSED matrix, logical [O, T]:
  * gvals [O, T/2], gmeta (see top).  dense_q_out (nullable, FP8 only): E5M2(fl32(dY * gscale)) [T, O].
  */
 sste_status sste_mvue_sparsify(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt,
-                               uint64_t seed, uint32_t tensor_id, uint32_t step,
+                               uint64_t seed, uint32_t tensor_id, uint32_t step, uint64_t token_offset,
                                const float *gscale_dev, sste_dtype odt,
                                void *gvals, void *gmeta, void *dense_q_out, void *stream);
 

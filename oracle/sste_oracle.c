@@ -373,7 +373,8 @@ void sste_oracle_mvue_group(const float a[4], float u, int pos[2], float val[2])
 
 /*
  * MVUE(dY^T): dY is [T, O] bf16 row-major; groups are 4 consecutive tokens of
- * one column j.  Group (j, tg) has global index g = tg*O + j; Philox counter
+ * one column j.  Group (j, tg) has global index g = (tg_offset + tg)*O + j (tg_offset = token groups
+ * that precede this dY in the whole batch; 0 unless the batch is sharded); Philox counter
  * (q_lo, q_hi, tensor_id, step) with q = g>>2, key (seed_lo, seed_hi); the group
  * uses output word g&3, top 24 bits, u = k * 2^-24.
  * Output is the canonical compressed format of the TRANSPOSED matrix: rows = O,
@@ -382,7 +383,7 @@ void sste_oracle_mvue_group(const float a[4], float u, int pos[2], float val[2])
  * theta (nullable) receives the uncast fp32 estimator, dense, as [T, O].
  */
 void sste_oracle_mvue(const uint16_t *dY, int T, int O, uint64_t seed, uint32_t tensor_id, uint32_t step,
-                      float gscale, int odt, void *gvals, uint16_t *gmeta, uint8_t *dense_q, float *theta)
+                      uint64_t tg_offset, float gscale, int odt, void *gvals, uint16_t *gmeta, uint8_t *dense_q, float *theta)
 {
     uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
 #pragma omp parallel for schedule(static)
@@ -390,7 +391,7 @@ void sste_oracle_mvue(const uint16_t *dY, int T, int O, uint64_t seed, uint32_t 
         for (int64_t tg = 0; tg < T / 4; ++tg) {
             float a[4];
             for (int i = 0; i < 4; ++i) a[i] = bf16_to_f32(dY[(4 * tg + i) * O + j]);
-            uint64_t g = (uint64_t)tg * (uint64_t)O + (uint64_t)j;
+            uint64_t g = (tg_offset + (uint64_t)tg) * (uint64_t)O + (uint64_t)j;
             uint64_t q = g >> 2;
             uint32_t ctr[4] = {(uint32_t)q, (uint32_t)(q >> 32), tensor_id, step};
             uint32_t rnd[4];

@@ -161,8 +161,12 @@ def mvue_group(a, u):
     return pos, val
 
 
-def mvue(dY, seed, tensor_id, step, odt=BF16, gscale=1.0, want_dense_q=False, want_theta=False):
-    """MVUE(dY^T) of a bf16 [T, O] gradient: canonical compressed [O, T/2] + meta [O, T/16]."""
+def mvue(dY, seed, tensor_id, step, odt=BF16, gscale=1.0, want_dense_q=False, want_theta=False, token_offset=0):
+    """MVUE(dY^T) of a bf16 [T, O] gradient: canonical compressed [O, T/2] + meta [O, T/16].
+
+    token_offset: tokens that precede this dY in the whole batch (the counter is the global group index).
+    """
+    assert token_offset % 4 == 0
     dY = _c(dY, np.uint16)
     T, O = dY.shape
     assert T % 16 == 0
@@ -172,7 +176,8 @@ def mvue(dY, seed, tensor_id, step, odt=BF16, gscale=1.0, want_dense_q=False, wa
     dense_q = np.empty((T, O), np.uint8) if want_dense_q else None
     theta = np.empty((T, O), np.float32) if want_theta else None
     lib().sste_oracle_mvue(_p(dY), T, O, ctypes.c_uint64(seed), ctypes.c_uint32(tensor_id),
-                           ctypes.c_uint32(step), ctypes.c_float(gscale), ctypes.c_int(odt),
+                           ctypes.c_uint32(step), ctypes.c_uint64(token_offset // 4), ctypes.c_float(gscale),
+                           ctypes.c_int(odt),
                            _p(gvals), _p(gmeta), _p(dense_q), _p(theta))
     return gvals, gmeta, dense_q, theta
 

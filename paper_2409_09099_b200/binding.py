@@ -114,11 +114,13 @@ class Context:
             self.handle, _ptr(X), T, _ptr(vals), _ptr(meta), O, I, _CODE_OF[X.dtype], _ptr(out_scale_dev),
             _ptr(Y), _CODE_OF[Y.dtype], _stream()))
 
-    def mvue_sparsify(self, dY, seed, tensor_id, step, gvals, gmeta, dense_q_out=None, gscale_dev=None):
+    def mvue_sparsify(self, dY, seed, tensor_id, step, gvals, gmeta, dense_q_out=None, gscale_dev=None,
+                      token_offset=0):
         T, O = dY.shape
         self._check(self.lib.sste_mvue_sparsify(
             self.handle, _ptr(dY), T, O, _CODE_OF[dY.dtype], ctypes.c_uint64(seed), ctypes.c_uint32(tensor_id),
-            ctypes.c_uint32(step), _ptr(gscale_dev), _CODE_OF[gvals.dtype], _ptr(gvals), _ptr(gmeta),
+            ctypes.c_uint32(step), ctypes.c_uint64(token_offset), _ptr(gscale_dev), _CODE_OF[gvals.dtype],
+            _ptr(gvals), _ptr(gmeta),
             _ptr(dense_q_out), _stream()))
 
     def linear_bwd_input(self, dY, Wt_dense, dX, out_scale_dev=None):

@@ -325,7 +325,7 @@ __device__ __forceinline__ MvueGroup mvue_group(float a0, float a1, float a2, fl
 template <bool FP8>
 __global__ void __launch_bounds__(EW_THREADS)
 mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t key1, uint32_t tensor_id,
-            uint32_t step, const float *__restrict__ gscale_dev, void *__restrict__ gvals,
+            uint32_t step, uint64_t tg_offset, const float *__restrict__ gscale_dev, void *__restrict__ gvals,
             uint8_t *__restrict__ gmeta, void *__restrict__ dense_q)
 {
     // bf16: 128 rows x 32 words; fp8: 128 rows x 16 words
@@ -346,7 +346,7 @@ mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t 
 #pragma unroll
         for (int i = 0; i < 4; ++i) in[i] = __ldg(dY + (tok0 + i) * row_chunks + jb * 16 + jc);
 
-        const uint64_t g0 = (static_cast<uint64_t>(tb) * 32 + tgl) * static_cast<uint64_t>(O) +
+        const uint64_t g0 = (tg_offset + static_cast<uint64_t>(tb) * 32 + tgl) * static_cast<uint64_t>(O) +
                             static_cast<uint64_t>(jb) * 128 + jc * 8;
         const uint64_t q = g0 >> 2;
         uint32_t rnd[8];
@@ -562,14 +562,15 @@ extern "C" sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O
 }
 
 extern "C" sste_status sste_mvue_sparsify(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt, uint64_t seed,
-                                          uint32_t tensor_id, uint32_t step, const float *gscale_dev, sste_dtype odt,
-                                          void *gvals, void *gmeta, void *dense_q_out, void *stream)
+                                          uint32_t tensor_id, uint32_t step, uint64_t token_offset,
+                                          const float *gscale_dev, sste_dtype odt, void *gvals, void *gmeta,
+                                          void *dense_q_out, void *stream)
 {
     if (!ctx || !dY || !gvals || !gmeta) return SSTE_ERR_INVALID_ARG;
     if (gdt != SSTE_BF16 || (odt != SSTE_BF16 && odt != SSTE_E5M2)) return SSTE_ERR_DTYPE;
     if (odt == SSTE_E5M2 && !gscale_dev) return SSTE_ERR_INVALID_ARG;
     if (odt == SSTE_BF16 && dense_q_out) return SSTE_ERR_INVALID_ARG;
-    if (!sste_mult128(O) || !sste_mult128(T)) return SSTE_ERR_SHAPE;
+    if (!sste_mult128(O) || !sste_mult128(T) || (token_offset % 4) != 0) return SSTE_ERR_SHAPE;
     if (!sste_aligned(dY, 128) || !sste_aligned(gvals, 128) || !sste_aligned(gmeta, 128) ||
         !sste_aligned(dense_q_out, 128))
         return SSTE_ERR_ALIGN;
@@ -580,11 +581,12 @@ extern "C" sste_status sste_mvue_sparsify(sste_ctx *ctx, const void *dY, int T, 
     const uint32_t key0 = static_cast<uint32_t>(seed), key1 = static_cast<uint32_t>(seed >> 32);
     if (odt == SSTE_E5M2)
         mvue_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(dY), O, T, key0, key1, tensor_id,
-                                                       step, gscale_dev, gvals, static_cast<uint8_t *>(gmeta),
-                                                       dense_q_out);
+                                                       step, token_offset / 4, gscale_dev, gvals,
+                                                       static_cast<uint8_t *>(gmeta), dense_q_out);
     else
         mvue_kernel<false><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(dY), O, T, key0, key1, tensor_id,
-                                                        step, nullptr, gvals, static_cast<uint8_t *>(gmeta), nullptr);
+                                                        step, token_offset / 4, nullptr, gvals,
+                                                        static_cast<uint8_t *>(gmeta), nullptr);
     return launch_result();
 }
 

@@ -88,10 +88,10 @@ class SsteLinear:
         return self.Y
 
     # (2b) backward: MVUE on the output gradient for grad_W, dense product for grad_X
-    def backward(self, dY, step: int = 0):
+    def backward(self, dY, step: int = 0, token_offset: int = 0):
         c = self.ctx
         if not self.fp8:
-            c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta)
+            c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta, token_offset=token_offset)
             c.linear_bwd_weight(self.gvals, self.gmeta, self.X, self.dW)
             c.linear_bwd_input(dY, self.w_dense, self.dX)
             self.launches += 3
@@ -99,7 +99,7 @@ class SsteLinear:
         c.amax(dY, self.amax[2:3])
         c.fp8_scale(self.amax[2:3], B.E5M2, self.scale[2:3], self.inv[2:3])
         c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta, dense_q_out=self.dYq,
-                        gscale_dev=self.scale[2:3])
+                        gscale_dev=self.scale[2:3], token_offset=token_offset)
         c.scalar_mul(self.inv[2:3], self.inv[0:1], self.inv_gx)
         c.scalar_mul(self.inv[2:3], self.inv[1:2], self.inv_gw)
         c.linear_bwd_weight(self.gvals, self.gmeta, self.Xq, self.dW, out_scale_dev=self.inv_gx)

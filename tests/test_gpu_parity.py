@@ -105,6 +105,17 @@ def test_mvue_sparsify(ctx, O, I, T):
     ctx.mvue_sparsify(dbf16(dY), seed, tid, step + 1, gvals2, gmeta2)
     assert not torch.equal(gmeta2, gmeta)
     assert np.array_equal(bits16(gvals2), orc.mvue(dY, seed, tid, step + 1)[0])
+    # a data-parallel shard: the counter starts at the shard's first token, so the two halves of the
+    # batch sparsified separately reproduce the unsharded result
+    if T % 256 == 0:
+        h = T // 2
+        for t0 in (0, h):
+            gv, gm = ctx.alloc_compressed(O, h)
+            ctx.mvue_sparsify(dbf16(dY[t0:t0 + h].copy()), seed, tid, step, gv, gm, token_offset=t0)
+            assert np.array_equal(bits16(gv), ogv[:, t0 // 2:(t0 + h) // 2])
+            assert np.array_equal(bits16(gv), orc.mvue(dY[t0:t0 + h].copy(), seed, tid, step, token_offset=t0)[0])
+    with pytest.raises(B.SsteError):
+        ctx.mvue_sparsify(dbf16(dY), seed, tid, step, gvals, gmeta, token_offset=2)
 
 
 @pytest.fixture(params=[0, 128, 192, 256])
