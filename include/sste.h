@@ -166,6 +166,28 @@ sste_status sste_linear_bwd_weight(sste_ctx *ctx, const void *gvals, const void 
                                    sste_dtype gdt, const void *X, int I, sste_dtype xdt,
                                    const float *out_scale_dev, void *dW, sste_dtype dwdt, void *stream);
 
+/*
+ * The same beta as sste_beta_init, for callers that cannot allocate device memory at all (the paper has
+ * no counterpart of this call; it exists for deployment).  A serving or training runtime that owns the
+ * whole memory pool, a plug-in that is handed only its inputs and outputs, or a job on a full device has
+ * no workspace to lend and therefore no sste_ctx.  This call needs neither: its reduction scratch is a
+ * fixed array inside the library image (about 129 KB that every GPU loading the library holds until the
+ * process exits).  It calls no cudaMalloc / cudaFree or other allocating routine.
+ *   device   ordinal of the GPU that W and beta_dev live on (made current for the call).
+ *   W        bf16 [O, I], O and I multiples of 128.  One partial per 128 x 128 tile is kept, and the array
+ *            holds 8192 of them: (O/128)*(I/128) > 8192 returns SSTE_ERR_WORKSPACE and launches nothing.
+ *   beta_dev device float, written asynchronously on `stream`.  If S_soft(W) is identically zero it
+ *            receives 1.0 (there is no context, so no status word records it).
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress); make that first
+ * call outside any stream capture.  All calls on a device share the one array: each call clears the ticket
+ * counter it needs at zero and overwrites the partials, so results never depend on earlier calls, but two
+ * calls whose kernels overlap on the GPU (different streams without ordering) race.  Sums are combined in
+ * tile order: the result is reproducible, and equals sste_beta_init up to the rounding of a different
+ * summation order (about 1e-7 relative).
+ */
+sste_status sste_beta_init_static(int device, const void *W, int O, int I, sste_dtype wdt, float *beta_dev,
+                                  void *stream);
+
 /* ---- FP8 whole-process variant (Sec. 5.2): per-tensor rescaling before the cast ---- */
 
 /* *amax_dev = max |x| over n bf16 elements (n % 8 == 0).  Exact, order-free.  The call first sets

@@ -27,7 +27,7 @@ EXPORTS = [
     "sste_vals_bytes", "sste_meta_bytes", "sste_beta_init", "sste_project_compress", "sste_linear_fwd",
     "sste_mvue_sparsify", "sste_linear_bwd_input", "sste_linear_bwd_weight", "sste_amax", "sste_fp8_scale",
     "sste_quantize_fp8", "sste_scalar_mul", "sste_meta_to_canonical", "sste_debug_force_tile_width", "sste_debug_force_splits",
-    "sste_workspace_bytes_recommended",
+    "sste_workspace_bytes_recommended", "sste_beta_init_static",
 ]
 
 
@@ -65,6 +65,20 @@ def _ptr(t):
 
 def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def beta_init_static(W, beta_dev):
+    """sste_beta_init_static: beta for callers that cannot lend a device workspace.
+
+    Needs no Context and allocates nothing on the device: the reduction scratch is a fixed array inside
+    libsste.so.  Same arguments as Context.beta_init; W may have at most 8192 tiles of 128 x 128.
+    Raises SsteError (code ERR_WORKSPACE for a tensor beyond that limit).
+    """
+    lib = load()
+    O, I = W.shape
+    st = lib.sste_beta_init_static(W.device.index or 0, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev), _stream())
+    if st != OK:
+        raise SsteError(st, lib.sste_status_string(st).decode())
 
 
 class Context:

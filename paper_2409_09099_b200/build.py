@@ -10,7 +10,7 @@ HERE = Path(__file__).resolve().parent
 ROOT = HERE.parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libsste.so"
-SOURCES = ["api.cu", "elementwise.cu", "gemm.cu"]
+SOURCES = ["api.cu", "elementwise.cu", "gemm.cu", "no_alloc.cu"]
 
 
 def _nvcc() -> str:
