@@ -247,9 +247,9 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 
 // Shared-memory / tensor-memory plan of one CTA for a tile of 256 x BN.  A stage holds 128 bytes of K per
 // A row and, for the sparse kernels, two B sub-tiles of 128 bytes of K each (the compressed A row covers
-// twice the K of one B row); the dense kernel pairs it with one B sub-tile.  BN = 256 fills the
-// accumulator half of tensor memory with one buffer; BN <= 192 leaves room for two, so the epilogue of a
-// tile overlaps the next tile's main loop.
+// twice the K of one B row); the dense kernel pairs it with one B sub-tile.  A sparse tile of BN = 256
+// leaves room for one accumulator buffer beside the metadata regions in the 512 tensor-memory columns;
+// BN <= 192, and every dense tile, has two, so the epilogue of a tile overlaps the next tile's main loop.
 template <bool SPARSE, int BN>
 struct Cfg {
     static constexpr int A_STAGE = 16384;                        // 128 rows x 128 bytes
@@ -258,11 +258,11 @@ struct Cfg {
     static constexpr int STAGE = A_STAGE + B_STAGE;
     static constexpr int FIT = (232448 - 1024 - 512 - STAGING_BYTES) / STAGE;   // 227 KB of shared memory per CTA
     static constexpr int STAGES = FIT > 8 ? 8 : FIT;
-    static constexpr int ACC_BUFS = (BN <= 192) ? 2 : 1;
+    static constexpr int ACC_BUFS = (!SPARSE || BN <= 192) ? 2 : 1;   // the dense kernel keeps no metadata in TMEM
     static constexpr int META_COL0 = ACC_BUFS * BN;              // metadata regions follow the accumulators
     static constexpr int THREADS = SPARSE ? 320 : 192;           // + 4 metadata warps for the sparse kernels
     static constexpr int SMEM_BYTES = STAGES * STAGE + STAGING_BYTES + 1024 /* alignment slack */ + 512 /* barriers */;
-    static_assert(META_COL0 + META_REGIONS * 16 <= TMEM_COLS, "tensor memory budget");
+    static_assert(META_COL0 + (SPARSE ? META_REGIONS * 16 : 0) <= TMEM_COLS, "tensor memory budget");
     static_assert(STAGES >= 3, "pipeline depth");
 };
 
