@@ -95,6 +95,17 @@ def oracle_step(tensors, seed, step, fp8=False):
     """One pass of the path on the CPU oracle for a list of (W, X, dY, beta32) samples."""
     from oracle import sste_oracle as orc
     for li, (W, X, dY, beta32) in enumerate(tensors):
+        if fp8:   # whole-process FP8: per-tensor scales, E4M3 forward operands, E5M2 gradient
+            _, _, wt = orc.project_compress(W, beta32)
+            sw, sx, sg = (orc.fp8_scale(orc.amax(wt), orc.E4M3), orc.fp8_scale(orc.amax(X), orc.E4M3),
+                          orc.fp8_scale(orc.amax(dY), orc.E5M2))
+            vals, meta, dense = orc.project_compress(W, beta32, odt=orc.E4M3, wscale=sw)
+            Xq = orc.quantize(X, sx, orc.E4M3)
+            orc.linear_fwd(Xq, orc.E4M3, vals, meta, orc.E4M3, 1.0 / (float(sx) * float(sw)))
+            gv, gm, dq, _ = orc.mvue(dY, seed, li, step, odt=orc.E5M2, gscale=sg, want_dense_q=True)
+            orc.linear_bwd_weight(gv, gm, orc.E5M2, Xq, orc.E4M3, 1.0 / (float(sg) * float(sx)))
+            orc.linear_bwd_input(dq, orc.E5M2, dense, orc.E4M3, 1.0 / (float(sg) * float(sw)))
+            continue
         vals, meta, dense = orc.project_compress(W, beta32)
         orc.linear_fwd(X, orc.BF16, vals, meta, orc.BF16)
         gv, gm, _, _ = orc.mvue(dY, seed, li, step)
@@ -118,10 +129,10 @@ def oracle_sample(cfg_id: int, tokens: int):
 def time_oracle(cfg_id: int, tokens: int, steps: int, warmup: int):
     cfg, tensors, flops = oracle_sample(cfg_id, tokens)
     for w in range(warmup):
-        oracle_step(tensors, cfg["seed"], w)
+        oracle_step(tensors, cfg["seed"], w, cfg["fp8"])
     t0 = time.perf_counter()
     for s in range(steps):
-        oracle_step(tensors, cfg["seed"], s)
+        oracle_step(tensors, cfg["seed"], s, cfg["fp8"])
     dt = (time.perf_counter() - t0) / max(steps, 1)
     cores = len(os.sched_getaffinity(0))
     return dict(value=flops / dt / 1e12, unit=UNIT, cores=cores, kind="oracle",
@@ -246,8 +257,6 @@ def run_gpu(args):
             step(args.warmup)
         graph.replay()
         torch.cuda.synchronize()
-    launches_before = sum(l.launches for l, _, _ in layers)
-    launches_per_step = None
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -268,7 +277,7 @@ def run_gpu(args):
     barrier()
     # second timed pass, eager, with an event between kernels: the per-kernel breakdown and roofline
     per_kernel = {k: [] for k in KERNELS}
-    n_before = sum(l.launches for l, _, _ in layers)
+    n_before = B.launch_count()                         # the library counts its own kernel launches
     for s in range(args.steps):
         flush.zero_()
         ev = []
@@ -279,10 +288,10 @@ def run_gpu(args):
                 base = li * 6
                 for ki, k in enumerate(KERNELS):
                     per_kernel[k].append((li, ev[base + ki].elapsed_time(ev[base + ki + 1])))
-    launches_per_step = (sum(l.launches for l, _, _ in layers) - n_before) // args.steps
+    launches_per_step = (B.launch_count() - n_before) // args.steps
     barrier()
     clocks = sampler.stop()
-    gpu_launches = launches_per_step * args.steps       # kernels executed inside the timed region
+    gpu_launches = launches_per_step * args.steps       # libsste kernels executed in the K timed steps
     total_ms = sum(step_ms)
     if world > 1:
         t = torch.tensor([total_ms], dtype=torch.float64, device=dev)

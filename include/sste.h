@@ -211,6 +211,11 @@ sste_status sste_scalar_mul(sste_ctx *ctx, const float *a_dev, const float *b_de
 sste_status sste_meta_to_canonical(sste_ctx *ctx, const void *meta, int rows, int k, sste_dtype dt,
                                    void *canonical_out, void *stream);
 
+/* Number of kernels this library has launched in the process so far (all entry points, all contexts; a
+ * product that splits its reduction counts its second pass too).  A benchmark reports the difference
+ * around its timed region. */
+unsigned long long sste_debug_launch_count(void);
+
 /* The three products pick the width of their output tiles (128, 192 or 256 columns) from the problem
  * shape.  This process-wide hook pins it so that tests can cover every variant; widths a product does
  * not support (192 needs a K-major B operand, i.e. the forward) fall back to the automatic choice.

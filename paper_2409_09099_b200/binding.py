@@ -27,7 +27,7 @@ EXPORTS = [
     "sste_vals_bytes", "sste_meta_bytes", "sste_beta_init", "sste_project_compress", "sste_linear_fwd",
     "sste_mvue_sparsify", "sste_linear_bwd_input", "sste_linear_bwd_weight", "sste_amax", "sste_fp8_scale",
     "sste_quantize_fp8", "sste_scalar_mul", "sste_meta_to_canonical", "sste_debug_force_tile_width", "sste_debug_force_splits",
-    "sste_workspace_bytes_recommended", "sste_beta_init_static",
+    "sste_workspace_bytes_recommended", "sste_beta_init_static", "sste_debug_launch_count",
 ]
 
 
@@ -65,6 +65,13 @@ def _ptr(t):
 
 def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def launch_count() -> int:
+    """Kernels launched by the library in this process so far (sste_debug_launch_count)."""
+    lib = load()
+    lib.sste_debug_launch_count.restype = ctypes.c_ulonglong
+    return int(lib.sste_debug_launch_count())
 
 
 def beta_init_static(W, beta_dev):

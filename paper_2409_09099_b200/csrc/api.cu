@@ -3,6 +3,12 @@
 
 #include "common.cuh"
 
+#include <atomic>
+
+static std::atomic<unsigned long long> g_launch_count{0};
+void sste_count_launches(int n) { g_launch_count.fetch_add(static_cast<unsigned long long>(n), std::memory_order_relaxed); }
+extern "C" unsigned long long sste_debug_launch_count(void) { return g_launch_count.load(std::memory_order_relaxed); }
+
 extern "C" size_t sste_workspace_bytes(void) { return SSTE_WS_BYTES; }
 extern "C" size_t sste_workspace_bytes_recommended(void) { return SSTE_WS_RECOMMENDED_BYTES; }
 

@@ -86,5 +86,8 @@ __device__ __host__ __forceinline__ uint32_t sste_meta_atom_byte16(uint32_t m, u
 }
 __device__ __host__ __forceinline__ uint32_t sste_meta_atom_byte8(uint32_t m, uint32_t k) { return 16u * m + (k >> 3); }
 
+// Process-wide count of kernels this library has launched (read by sste_debug_launch_count).
+void sste_count_launches(int n);
+
 // entry points implemented in the other translation units
 sste_status sste_gemm_launch_check(const sste_ctx *ctx);

@@ -513,7 +513,13 @@ int grid_for(size_t work_items, int sm_count)
     return static_cast<int>(blocks);
 }
 
-sste_status launch_result() { return cudaGetLastError() == cudaSuccess ? SSTE_OK : SSTE_ERR_CUDA; }
+// every entry point of this file launches exactly one kernel
+sste_status launch_result()
+{
+    if (cudaGetLastError() != cudaSuccess) return SSTE_ERR_CUDA;
+    sste_count_launches(1);
+    return SSTE_OK;
+}
 
 }  // namespace
 

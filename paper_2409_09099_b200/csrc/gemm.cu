@@ -799,7 +799,9 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
             pp.partials, p.M, p.N, BN, pp.splits, m_tiles, pp.split_from, n_split_tiles, p.out_scale,
             static_cast<uint4 *>(p.D));
     }
-    return cudaGetLastError() == cudaSuccess ? SSTE_OK : SSTE_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return SSTE_ERR_CUDA;
+    sste_count_launches(pp.splits > 1 ? 2 : 1);
+    return SSTE_OK;
 }
 
 int g_force_splits = 0;   // test hook: 0 = automatic split-K factor
