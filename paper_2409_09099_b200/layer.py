@@ -89,20 +89,44 @@ class SsteLinear:
 
     # (2b) backward: MVUE on the output gradient for grad_W, dense product for grad_X
     def backward(self, dY, step: int = 0, token_offset: int = 0):
+        self.sparsify_grad(dY, step, token_offset)
+        self.grad_weight()
+        self.grad_input(dY)
+        return self.dX, self.dW
+
+    # (2b.1) MVUE(dY^T): 2:4 along tokens, compressed and transposed for the grad_W product
+    def sparsify_grad(self, dY, step: int = 0, token_offset: int = 0):
         c = self.ctx
         if not self.fp8:
             c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta, token_offset=token_offset)
-            c.linear_bwd_weight(self.gvals, self.gmeta, self.X, self.dW)
-            c.linear_bwd_input(dY, self.w_dense, self.dX)
-            self.launches += 3
-            return self.dX, self.dW
+            self.launches += 1
+            return
         c.amax(dY, self.amax[2:3])
         c.fp8_scale(self.amax[2:3], B.E5M2, self.scale[2:3], self.inv[2:3])
         c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta, dense_q_out=self.dYq,
                         gscale_dev=self.scale[2:3], token_offset=token_offset)
+        self.launches += 3
+
+    # (2b.2) grad_W = MVUE(dY^T) X, sparse
+    def grad_weight(self):
+        c = self.ctx
+        if not self.fp8:
+            c.linear_bwd_weight(self.gvals, self.gmeta, self.X, self.dW)
+            self.launches += 1
+            return self.dW
         c.scalar_mul(self.inv[2:3], self.inv[0:1], self.inv_gx)
-        c.scalar_mul(self.inv[2:3], self.inv[1:2], self.inv_gw)
         c.linear_bwd_weight(self.gvals, self.gmeta, self.Xq, self.dW, out_scale_dev=self.inv_gx)
+        self.launches += 2
+        return self.dW
+
+    # (2b.3) grad_X = dY w~, dense
+    def grad_input(self, dY):
+        c = self.ctx
+        if not self.fp8:
+            c.linear_bwd_input(dY, self.w_dense, self.dX)
+            self.launches += 1
+            return self.dX
+        c.scalar_mul(self.inv[2:3], self.inv[1:2], self.inv_gw)
         c.linear_bwd_input(self.dYq, self.w_dense, self.dX, out_scale_dev=self.inv_gw)
-        self.launches += 7
-        return self.dX, self.dW
+        self.launches += 2
+        return self.dX
