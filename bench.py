@@ -389,6 +389,7 @@ def run_gpu(args):
                     "ms_per_step": e2e_ms},
             "gpu_launches": gpu_launches,
             "roofline": roofline,
+            "rooflines": rooflines,
             "kernels": breakdown,
             "cpu_baseline": cpu_base,
             "device_status": status,
