@@ -86,6 +86,33 @@ __device__ __host__ __forceinline__ uint32_t sste_meta_atom_byte16(uint32_t m, u
 }
 __device__ __host__ __forceinline__ uint32_t sste_meta_atom_byte8(uint32_t m, uint32_t k) { return 16u * m + (k >> 3); }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of the path is launched with programmatic stream serialisation: its CTAs may be scheduled,
+// and run their prologue (barrier and tensor-memory set-up, descriptor prefetch, index arithmetic), while the
+// previous kernel of the stream is still draining.  sste_pdl_wait() returns once that previous kernel has
+// finished and its writes are visible; no kernel touches global memory before it.  sste_pdl_trigger(), issued
+// first thing, is what lets the NEXT kernel of the stream be scheduled early (it takes effect when every CTA
+// of this grid has issued it or exited, so the successor never competes with CTAs not yet started).
+__device__ __forceinline__ void sste_pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void sste_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t sste_launch(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                               Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // Process-wide count of kernels this library has launched (read by sste_debug_launch_count).
 void sste_count_launches(int n);
 

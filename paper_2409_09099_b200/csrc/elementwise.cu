@@ -75,6 +75,8 @@ project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restr
     __shared__ __align__(16) uint8_t meta_s[512];
     const int tid = threadIdx.x;
     const int kb = blockIdx.x, rb = blockIdx.y;
+    sste_pdl_trigger();
+    sste_pdl_wait();
     const float beta = *beta_dev;
     const float wscale = FP8 ? *wscale_dev : 1.0f;
     const size_t row_chunks = static_cast<size_t>(I) / 8;
@@ -168,6 +170,8 @@ beta_kernel(const uint4 *__restrict__ W, size_t n_chunks, double *__restrict__ p
 {
     __shared__ double red[2][EW_THREADS / 32];
     __shared__ bool is_last;
+    sste_pdl_trigger();
+    sste_pdl_wait();
     double num = 0.0, den = 0.0;
     for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
          c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
@@ -333,6 +337,8 @@ mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t 
     __shared__ __align__(16) uint8_t meta_s[2048];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int jb = blockIdx.x, tb = blockIdx.y;   // column block, token block
+    sste_pdl_trigger();
+    sste_pdl_wait();
     const float gscale = FP8 ? *gscale_dev : 1.0f;
     const size_t row_chunks = static_cast<size_t>(O) / 8;
 
@@ -434,6 +440,8 @@ __global__ void __launch_bounds__(EW_THREADS)
 amax_kernel(const uint4 *__restrict__ x, size_t n_chunks, float *__restrict__ amax_dev)
 {
     uint32_t best = 0;   // magnitude bits of bf16 compare like unsigned integers
+    sste_pdl_trigger();
+    sste_pdl_wait();
     for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
          c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
         const uint4 v = __ldg(x + c);
@@ -452,19 +460,28 @@ amax_kernel(const uint4 *__restrict__ x, size_t n_chunks, float *__restrict__ am
 
 __global__ void fp8_scale_kernel(const float *amax_dev, float fp8_max, float *scale_dev, float *inv_scale_dev)
 {
+    sste_pdl_trigger();
+    sste_pdl_wait();
     const float a = *amax_dev;
     const float s = (a == 0.0f) ? 1.0f : __fdiv_rn(fp8_max, a);
     *scale_dev = s;
     if (inv_scale_dev) *inv_scale_dev = __fdiv_rn(1.0f, s);
 }
 
-__global__ void scalar_mul_kernel(const float *a, const float *b, float *out) { *out = __fmul_rn(*a, *b); }
+__global__ void scalar_mul_kernel(const float *a, const float *b, float *out)
+{
+    sste_pdl_trigger();
+    sste_pdl_wait();
+    *out = __fmul_rn(*a, *b);
+}
 
 template <bool E5M2>
 __global__ void __launch_bounds__(EW_THREADS)
 quantize_kernel(const uint4 *__restrict__ x, size_t n_chunks, const float *__restrict__ scale_dev,
                 uint2 *__restrict__ q)
 {
+    sste_pdl_trigger();
+    sste_pdl_wait();
     const float scale = *scale_dev;
     for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
          c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
@@ -489,6 +506,8 @@ template <bool EIGHT_BIT>
 __global__ void __launch_bounds__(EW_THREADS)
 meta_to_canonical_kernel(const uint8_t *__restrict__ meta, int rows, int k, uint16_t *__restrict__ out)
 {
+    sste_pdl_trigger();
+    sste_pdl_wait();
     const size_t words = static_cast<size_t>(rows) * (k / 16);
     for (size_t w = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; w < words;
          w += static_cast<size_t>(gridDim.x) * EW_THREADS) {
@@ -536,8 +555,8 @@ extern "C" sste_status sste_beta_init(sste_ctx *ctx, const void *W, int O, int I
     if (!guard.ok) return SSTE_ERR_CUDA;
     const size_t n_chunks = static_cast<size_t>(O) * I / 8;
     const int grid = grid_for(n_chunks, ctx->sm_count);
-    beta_kernel<<<grid, EW_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint4 *>(W), n_chunks, ctx->partials_dev, ctx->counter_dev, beta_dev, ctx->status_dev);
+    sste_launch(beta_kernel, dim3(grid), dim3(EW_THREADS), 0, static_cast<cudaStream_t>(stream),
+                static_cast<const uint4 *>(W), n_chunks, ctx->partials_dev, ctx->counter_dev, beta_dev, ctx->status_dev);
     return launch_result();
 }
 
@@ -557,13 +576,11 @@ extern "C" sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O
     const dim3 grid(I / 128, O / PC_ROWS);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (odt == SSTE_E4M3)
-        project_compress_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(W), I, beta_dev,
-                                                                   wscale_dev, vals, static_cast<uint8_t *>(meta),
-                                                                   dense_out);
+        sste_launch(project_compress_kernel<true>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(W),
+                    I, beta_dev, wscale_dev, vals, static_cast<uint8_t *>(meta), dense_out);
     else
-        project_compress_kernel<false><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(W), I, beta_dev,
-                                                                    nullptr, vals, static_cast<uint8_t *>(meta),
-                                                                    dense_out);
+        sste_launch(project_compress_kernel<false>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(W),
+                    I, beta_dev, nullptr, vals, static_cast<uint8_t *>(meta), dense_out);
     return launch_result();
 }
 
@@ -586,13 +603,13 @@ extern "C" sste_status sste_mvue_sparsify(sste_ctx *ctx, const void *dY, int T, 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const uint32_t key0 = static_cast<uint32_t>(seed), key1 = static_cast<uint32_t>(seed >> 32);
     if (odt == SSTE_E5M2)
-        mvue_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(dY), O, T, key0, key1, tensor_id,
-                                                       step, token_offset / 4, gscale_dev, gvals,
-                                                       static_cast<uint8_t *>(gmeta), dense_q_out);
+        sste_launch(mvue_kernel<true>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(dY), O, T,
+                    key0, key1, tensor_id, step, token_offset / 4, gscale_dev, gvals, static_cast<uint8_t *>(gmeta),
+                    dense_q_out);
     else
-        mvue_kernel<false><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(dY), O, T, key0, key1, tensor_id,
-                                                        step, token_offset / 4, nullptr, gvals,
-                                                        static_cast<uint8_t *>(gmeta), nullptr);
+        sste_launch(mvue_kernel<false>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(dY), O, T,
+                    key0, key1, tensor_id, step, token_offset / 4, nullptr, gvals, static_cast<uint8_t *>(gmeta),
+                    nullptr);
     return launch_result();
 }
 
@@ -606,8 +623,8 @@ extern "C" sste_status sste_amax(sste_ctx *ctx, const void *x, size_t n, sste_dt
     if (!guard.ok) return SSTE_ERR_CUDA;
     const size_t n_chunks = n / 8;
     SSTE_CUDA_TRY(cudaMemsetAsync(amax_dev, 0, sizeof(float), static_cast<cudaStream_t>(stream)));
-    amax_kernel<<<grid_for(n_chunks, ctx->sm_count), EW_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint4 *>(x), n_chunks, amax_dev);
+    sste_launch(amax_kernel, dim3(grid_for(n_chunks, ctx->sm_count)), dim3(EW_THREADS), 0,
+                static_cast<cudaStream_t>(stream), static_cast<const uint4 *>(x), n_chunks, amax_dev);
     return launch_result();
 }
 
@@ -618,8 +635,8 @@ extern "C" sste_status sste_fp8_scale(sste_ctx *ctx, const float *amax_dev, sste
     if (odt != SSTE_E4M3 && odt != SSTE_E5M2) return SSTE_ERR_DTYPE;
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
-    fp8_scale_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(amax_dev, odt == SSTE_E4M3 ? 448.0f : 57344.0f,
-                                                                     scale_dev, inv_scale_dev);
+    sste_launch(fp8_scale_kernel, dim3(1), dim3(1), 0, static_cast<cudaStream_t>(stream), amax_dev,
+                odt == SSTE_E4M3 ? 448.0f : 57344.0f, scale_dev, inv_scale_dev);
     return launch_result();
 }
 
@@ -629,7 +646,7 @@ extern "C" sste_status sste_scalar_mul(sste_ctx *ctx, const float *a_dev, const 
     if (!ctx || !a_dev || !b_dev || !out_dev) return SSTE_ERR_INVALID_ARG;
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
-    scalar_mul_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(a_dev, b_dev, out_dev);
+    sste_launch(scalar_mul_kernel, dim3(1), dim3(1), 0, static_cast<cudaStream_t>(stream), a_dev, b_dev, out_dev);
     return launch_result();
 }
 
@@ -646,11 +663,11 @@ extern "C" sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n,
     const int grid = grid_for(n_chunks, ctx->sm_count);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (odt == SSTE_E5M2)
-        quantize_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(x), n_chunks, scale_dev,
-                                                           static_cast<uint2 *>(q));
+        sste_launch(quantize_kernel<true>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(x),
+                    n_chunks, scale_dev, static_cast<uint2 *>(q));
     else
-        quantize_kernel<false><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint4 *>(x), n_chunks, scale_dev,
-                                                            static_cast<uint2 *>(q));
+        sste_launch(quantize_kernel<false>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(x),
+                    n_chunks, scale_dev, static_cast<uint2 *>(q));
     return launch_result();
 }
 
@@ -665,10 +682,10 @@ extern "C" sste_status sste_meta_to_canonical(sste_ctx *ctx, const void *meta, i
     const int grid = grid_for(words, ctx->sm_count);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (dt == SSTE_BF16)
-        meta_to_canonical_kernel<false><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint8_t *>(meta), rows, k,
-                                                                     static_cast<uint16_t *>(canonical_out));
+        sste_launch(meta_to_canonical_kernel<false>, dim3(grid), dim3(EW_THREADS), 0, s,
+                    static_cast<const uint8_t *>(meta), rows, k, static_cast<uint16_t *>(canonical_out));
     else
-        meta_to_canonical_kernel<true><<<grid, EW_THREADS, 0, s>>>(static_cast<const uint8_t *>(meta), rows, k,
-                                                                    static_cast<uint16_t *>(canonical_out));
+        sste_launch(meta_to_canonical_kernel<true>, dim3(grid), dim3(EW_THREADS), 0, s,
+                    static_cast<const uint8_t *>(meta), rows, k, static_cast<uint16_t *>(canonical_out));
     return launch_result();
 }

@@ -232,7 +232,14 @@ int g_probe_mode = 0;
 long long *g_probe_dbg = nullptr;
 #define PROBE_MODE(p) ((p).probe)
 #define PROBE_STAMP(p, tile, k) do { if ((p).dbg && blockIdx.x == 0 && (tile) < 16) (p).dbg[(tile) * 4 + (k)] = clock64(); } while (0)
+// kernel-level stamps: [64 + k] = clock64 of CTA 0, [72 + k] = globaltimer of CTA 0, [80] / [81] = min entry / max exit (ns) over CTAs
+__device__ __forceinline__ long long probe_gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define PROBE_KSTAMP(p, k) do { if ((p).dbg && threadIdx.x == 0) { long long g__ = probe_gtime(); \
+    if (blockIdx.x == 0) { (p).dbg[64 + (k)] = clock64(); (p).dbg[72 + (k)] = g__; } \
+    if ((k) == 0) atomicMin(reinterpret_cast<unsigned long long *>((p).dbg + 80), static_cast<unsigned long long>(g__)); \
+    if ((k) == 2) atomicMax(reinterpret_cast<unsigned long long *>((p).dbg + 81), static_cast<unsigned long long>(g__)); } } while (0)
 #else
+#define PROBE_KSTAMP(p, k) do { } while (0)
 #define PROBE_MODE(p) 0
 #define PROBE_STAMP(p, tile, k) do { } while (0)
 #endif
@@ -274,6 +281,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_p,
             const uint8_t *__restrict__ meta, const GemmParams p)
 {
+    sste_pdl_trigger();
+    PROBE_KSTAMP(p, 0);
     using C = Cfg<SPARSE, BN>;
     constexpr int NS = C::STAGES;
     constexpr int NB = C::ACC_BUFS;
@@ -351,6 +360,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     __syncthreads();
     cluster_sync();          // the peer's barriers are initialised before anything signals them
     tc_fence_after();
+    sste_pdl_wait();         // everything above overlapped the previous kernel; global memory from here on
+    PROBE_KSTAMP(p, 1);
     const uint32_t tmem_base = *tmem_slot_ptr;
 
     if (warp == 0) {
@@ -679,6 +690,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
+    PROBE_KSTAMP(p, 2);
 }
 
 // ------------------------------------------------------------------ host side
@@ -709,8 +721,10 @@ __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, int splits, int m_tiles, int split_from,
                      int n_split_tiles, const float *__restrict__ out_scale, uint4 *__restrict__ out)
 {
+    sste_pdl_trigger();
     const int vec_per_row = bn / 8;
     const size_t vecs = static_cast<size_t>(n_split_tiles) * 2 * BM * vec_per_row;
+    sste_pdl_wait();
     const float scale = out_scale ? *out_scale : 1.0f;
     for (size_t v = static_cast<size_t>(blockIdx.x) * 256 + threadIdx.x; v < vecs; v += static_cast<size_t>(gridDim.x) * 256) {
         const int col = static_cast<int>(v % vec_per_row) * 8;
@@ -790,14 +804,17 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         !make_map(ctx, &map_p, pp.partials, 4, static_cast<uint64_t>(n_split_tiles) * 2 * pp.splits * BM, BN, 32, BM,
                   CU_TENSOR_MAP_SWIZZLE_128B))
         return SSTE_ERR_CUDA;
-    kern<<<2 * pairs, C::THREADS, C::SMEM_BYTES, stream>>>(map_a, map_b, map_d, map_p, static_cast<const uint8_t *>(meta), pp);
+    if (sste_launch(kern, dim3(2 * pairs), dim3(C::THREADS), C::SMEM_BYTES, stream, map_a, map_b, map_d, map_p,
+                    static_cast<const uint8_t *>(meta), pp) != cudaSuccess)
+        return SSTE_ERR_CUDA;
     if (pp.splits > 1) {
         const size_t vecs = static_cast<size_t>(n_split_tiles) * 2 * BM * (BN / 8);
         size_t blocks = (vecs + 255) / 256;
         if (blocks > static_cast<size_t>(ctx->sm_count) * 16) blocks = static_cast<size_t>(ctx->sm_count) * 16;
-        splitk_reduce_kernel<<<static_cast<unsigned int>(blocks), 256, 0, stream>>>(
-            pp.partials, p.M, p.N, BN, pp.splits, m_tiles, pp.split_from, n_split_tiles, p.out_scale,
-            static_cast<uint4 *>(p.D));
+        if (sste_launch(splitk_reduce_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(256), 0, stream,
+                        pp.partials, p.M, p.N, BN, pp.splits, m_tiles, pp.split_from, n_split_tiles, p.out_scale,
+                        static_cast<uint4 *>(p.D)) != cudaSuccess)
+            return SSTE_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return SSTE_ERR_CUDA;
     sste_count_launches(pp.splits > 1 ? 2 : 1);
@@ -833,12 +850,20 @@ SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int alig
 }
 
 // Tile width, from timings on B200 over the GPT-2- and 7B-shaped layers: 256 columns is the fastest
-// almost everywhere (least L2 -> shared-memory traffic per flop); only the forward with a short
-// reduction (K <= 1024) gains from 192 columns, where the second accumulator buffer hides an
-// epilogue that is as long as the main loop.
-int pick_bn(bool b_k_major, int K)
+// almost everywhere (least L2 -> shared-memory traffic per flop); the forward gains from 192 columns
+// with a short reduction (K <= 1024), where the second accumulator buffer hides an epilogue that is as
+// long as the main loop, and when 256-wide tiles leave most of the last wave empty.
+int pick_bn(bool b_k_major, int M, int N, int K, int pairs)
 {
-    return (b_k_major && K <= 1024) ? 192 : 256;
+    if (!b_k_major) return 256;
+    if (K <= 1024) return 192;
+    // Longer reductions: 256 columns unless the tile count quantises badly (GPT-2 fc2 forward: 96 tiles on
+    // 74 CTA pairs are two waves; 129 tiles of 192 columns are two waves of 3/4 the work).  A 192-wide tile
+    // costs about 8 % more per flop (measured at many waves).
+    const long m_tiles = (M + 2 * BM - 1) / (2 * BM);
+    const long waves256 = (m_tiles * ((N + 255) / 256) + pairs - 1) / pairs;
+    const long waves192 = (m_tiles * ((N + 191) / 192) + pairs - 1) / pairs;
+    return (waves192 * 192 * 108 < waves256 * 256 * 100) ? 192 : 256;
 }
 
 bool fmt_code(sste_dtype dt, int *elt, uint32_t *code)
@@ -865,7 +890,7 @@ sste_status launch_out(const sste_ctx *ctx, const void *A, const void *B, const 
     cands[n++] = 256;
     if (!(MN && ELT == 1)) cands[n++] = 128;   // MN-major B: each CTA needs whole 128-byte chunks of N
     if (!MN) cands[n++] = 192;
-    int bn = pick_bn(!MN, p.K);
+    int bn = pick_bn(!MN, p.M, p.N, p.K, ctx->sm_count / 2);
     for (int i = 0; i < n; ++i)
         if (cands[i] == g_force_bn) bn = g_force_bn;
     if constexpr (!MN) {
