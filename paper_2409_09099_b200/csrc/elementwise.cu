@@ -244,11 +244,11 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 {
 #pragma unroll
     for (int round = 0; round < 10; ++round) {
-        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-        const uint32_t n0 = hi1 ^ c1 ^ k0;
-        const uint32_t n2 = hi0 ^ c3 ^ k1;
-        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        const uint64_t p0 = static_cast<uint64_t>(0xD2511F53u) * c0;   // one wide multiply gives both halves
+        const uint64_t p1 = static_cast<uint64_t>(0xCD9E8D57u) * c2;
+        const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ k1;
+        c0 = n0; c1 = static_cast<uint32_t>(p1); c2 = n2; c3 = static_cast<uint32_t>(p0);
         k0 += 0x9E3779B9u;
         k1 += 0xBB67AE85u;
     }
@@ -268,10 +268,14 @@ struct MvueGroup {
 //                            by the point u*rest on the others' cumulative sums, carries sign(a_j)*rest;
 //   unclipped (m_x <  rest): the points u*S/2 and u*S/2 + S/2 on the cumulative sums pick two elements,
 //                            both carry sign(a_j)*S/2.
-// Written with one-hot predicates and counting compares instead of index-driven selects (the kernel is
-// bound by the integer/fp32 pipes, not by HBM); every fp32 step is a single rounded operation.
-__device__ __forceinline__ MvueGroup mvue_group(float a0, float a1, float a2, float a3, float u)
+// The kernel is bound by instruction issue, not by HBM, so this is written for instruction count: no
+// branches, one-hot predicates, compares counted as 0 / -1 masks, and the two kept inputs picked by a byte
+// permute of the packed bf16 pairs p01 = a0 | a1 << 16, p23 = a2 | a3 << 16 (only their sign, or for the
+// clipped maximum their 16 bits, is needed).  Every fp32 step is a single rounded operation.
+__device__ __forceinline__ MvueGroup mvue_group(uint32_t p01, uint32_t p23, float u)
 {
+    const float a0 = __uint_as_float(p01 << 16), a1 = __uint_as_float(p01 & 0xffff0000u);
+    const float a2 = __uint_as_float(p23 << 16), a3 = __uint_as_float(p23 & 0xffff0000u);
     const float m0 = fabsf(a0), m1 = fabsf(a1), m2 = fabsf(a2), m3 = fabsf(a3);
     const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
     const bool e0 = (m0 == mx);
@@ -279,7 +283,6 @@ __device__ __forceinline__ MvueGroup mvue_group(float a0, float a1, float a2, fl
     const bool e2 = !e0 && !e1 && (m2 == mx);
     const bool e3 = !e0 && !e1 && !e2;
     const uint32_t xi = e0 ? 0u : e1 ? 1u : e2 ? 2u : 3u;
-    const float ax = e0 ? a0 : e1 ? a1 : e2 ? a2 : a3;
     // cumulative sums without x (adding +0 is exact) and with it
     const float z0 = e0 ? 0.0f : m0;
     const float z1 = __fadd_rn(z0, e1 ? 0.0f : m1);
@@ -293,29 +296,28 @@ __device__ __forceinline__ MvueGroup mvue_group(float a0, float a1, float a2, fl
     const float c0 = clipped ? z0 : m0, c1 = clipped ? z1 : s1, c2 = clipped ? z2 : s2;
     const float r1 = __fmul_rn(u, h);
     const float r2 = __fadd_rn(r1, h);
-    const uint32_t j1 = (c0 <= r1 ? 1u : 0u) + (c1 <= r1 ? 1u : 0u) + (c2 <= r1 ? 1u : 0u);
-    const uint32_t n2 = (c0 <= r2 ? 1u : 0u) + (c1 <= r2 ? 1u : 0u) + (c2 <= r2 ? 1u : 0u);
-    // index pair before ordering: (ia, ib) = (other, x) when clipped, (j1, j2) otherwise
-    uint32_t ia, ib;
-    if (clipped) {
-        ia = (rest == 0.0f) ? (e0 ? 1u : 0u) : j1;
-        ib = xi;
-    } else {
-        const bool tail = (j1 == 3u);
-        ia = tail ? 2u : j1;
-        ib = tail ? 3u : max(j1 + 1u, n2);
-    }
-    // candidates sign(a_i) * h; a zero h yields +0
+    // number of cumulative sums at or below each point: compares as 0 / -1, one three-input add each
+    const int j1 = -(((c0 <= r1) ? -1 : 0) + ((c1 <= r1) ? -1 : 0) + ((c2 <= r1) ? -1 : 0));
+    const int n2 = -(((c0 <= r2) ? -1 : 0) + ((c1 <= r2) ? -1 : 0) + ((c2 <= r2) ? -1 : 0));
+    // index pair before ordering: (other, x) when clipped; (j1, j2) otherwise, where a first point in the
+    // last element (j1 = 3) gives the pair (2, 3)
+    const int ia_c = (rest == 0.0f) ? (e0 ? 1 : 0) : j1;
+    const int ia_u = min(j1, 2);
+    const int ib_u = min(max(j1 + 1, n2), 3);
+    const uint32_t ia = static_cast<uint32_t>(clipped ? ia_c : ia_u);
+    const uint32_t ib = clipped ? xi : static_cast<uint32_t>(ib_u);
+    // bf16 bits of a_ia and a_ib in the upper half (lower half: don't care)
+    const uint32_t sa = __byte_perm(p01, p23, ia * 0x2200u + 0x1000u);
+    const uint32_t sb = __byte_perm(p01, p23, ib * 0x2200u + 0x1000u);
+    // kept values sign(a_i) * h; a zero h yields +0; the clipped maximum keeps its own value
     const uint32_t hb = __float_as_uint(h);
     const uint32_t sgn = (hb == 0u) ? 0u : 0x80000000u;
-    const float h0 = __uint_as_float((__float_as_uint(a0) & sgn) | hb), h1 = __uint_as_float((__float_as_uint(a1) & sgn) | hb);
-    const float h2 = __uint_as_float((__float_as_uint(a2) & sgn) | hb), h3 = __uint_as_float((__float_as_uint(a3) & sgn) | hb);
-    const float va = sel4(ia, h0, h1, h2, h3);
-    const float vb = clipped ? ax : sel4(ib, h0, h1, h2, h3);
+    const float va = __uint_as_float((sa & sgn) | hb);
+    const float vb = __uint_as_float(clipped ? (sb & 0xffff0000u) : ((sb & sgn) | hb));
     MvueGroup r;
     const bool swap = ia > ib;
-    r.q0 = swap ? ib : ia;
-    r.q1 = swap ? ia : ib;
+    r.q0 = min(ia, ib);
+    r.q1 = max(ia, ib);
     r.v0 = swap ? vb : va;
     r.v1 = swap ? va : vb;
     return r;
@@ -327,7 +329,7 @@ __device__ __forceinline__ MvueGroup mvue_group(float a0, float a1, float a2, fl
 // (8 groups, two Philox calls); results are transposed through shared memory so that every
 // output row (= column of dY) receives whole 128-byte lines.
 template <bool FP8>
-__global__ void __launch_bounds__(EW_THREADS)
+__global__ void __launch_bounds__(EW_THREADS, 4)
 mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t key1, uint32_t tensor_id,
             uint32_t step, uint64_t tg_offset, const float *__restrict__ gscale_dev, void *__restrict__ gvals,
             uint8_t *__restrict__ gmeta, void *__restrict__ dense_q)
@@ -367,25 +369,21 @@ mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t 
         uint32_t nibs = 0;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            float a[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t word = raw[i][e >> 1];
-                a[i] = sste_bf16_bits_to_f32((e & 1) ? (word >> 16) : (word & 0xffffu));
-            }
+            // the group of column e: one bf16 from each of the four token rows, packed in pairs
+            const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+            const uint32_t p01 = __byte_perm(raw[0][e >> 1], raw[1][e >> 1], sel);
+            const uint32_t p23 = __byte_perm(raw[2][e >> 1], raw[3][e >> 1], sel);
             const float u = __uint2float_rn(rnd[e] >> 8) * 0x1p-24f;
-            const MvueGroup r = mvue_group(a[0], a[1], a[2], a[3], u);
+            const MvueGroup r = mvue_group(p01, p23, u);
             nibs |= (r.q0 | (r.q1 << 2)) << (4 * e);
             const int jl = jc * 8 + e;
             if (FP8) {
-                const uint32_t b0 = sste_f32_to_e5m2(__fmul_rn(r.v0, gscale));
-                const uint32_t b1 = sste_f32_to_e5m2(__fmul_rn(r.v1, gscale));
-                reinterpret_cast<uint16_t *>(vals_s)[jl * 32 + (tgl ^ (8 * (jc & 3)))] =
-                    static_cast<uint16_t>(b0 | (b1 << 8));
+                const uint32_t pair = static_cast<uint32_t>(__nv_cvt_float2_to_fp8x2(
+                    make_float2(__fmul_rn(r.v0, gscale), __fmul_rn(r.v1, gscale)), __NV_SATFINITE, __NV_E5M2));
+                reinterpret_cast<uint16_t *>(vals_s)[jl * 32 + (tgl ^ (8 * (jc & 3)))] = static_cast<uint16_t>(pair);
             } else {
-                const uint32_t b0 = sste_f32_to_bf16_bits(r.v0);
-                const uint32_t b1 = sste_f32_to_bf16_bits(r.v1);
-                vals_s[jl * 32 + (tgl ^ (4 * (jc & 7)))] = b0 | (b1 << 16);
+                const __nv_bfloat162 pair = __floats2bfloat162_rn(r.v0, r.v1);
+                vals_s[jl * 32 + (tgl ^ (4 * (jc & 7)))] = *reinterpret_cast<const uint32_t *>(&pair);
             }
         }
         if (FP8 && dense_q) {
