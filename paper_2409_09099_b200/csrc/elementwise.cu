@@ -14,51 +14,45 @@ constexpr int PC_CHUNKS = PC_ROWS * 16 / EW_THREADS;         // 16-byte chunks p
 // ---------------------------------------------------------------- group of four: S_soft + kept pair
 
 struct SoftGroup {
-    float w[4];     // beta * S_soft, pruned entries +0
+    float w[4];       // beta * S_soft (times the FP8 scale), pruned entries +0
     uint32_t p0, p1;  // kept positions, p0 < p1
 };
 
-// bits[i]: bf16 bit pattern of a_i (low 16 bits)
+// w01 = a0 | a1 << 16, w23 = a2 | a3 << 16 (bf16 bit patterns).  Written for instruction count (the kernel
+// is bound by instruction issue): the threshold t = second-smallest magnitude comes from packed 16-bit
+// min/max on the magnitude bits (bf16 magnitudes order like unsigned integers), sign(a)(|a| - t) is the single
+// subtraction a - copysign(t, a), and the kept pair is the top two of four integer keys
+// (magnitude << 2 | 3 - index: magnitude descending, index ascending; pairwise distinct) found with a
+// seven-operation min/max network.
 template <bool FP8>
-__device__ __forceinline__ SoftGroup soft_group(const uint32_t bits[4], float beta, float wscale)
+__device__ __forceinline__ SoftGroup soft_group(uint32_t w01, uint32_t w23, float beta, float wscale)
 {
     SoftGroup r;
-    float a[4], m[4];
-    uint32_t key[4];
+    const uint32_t m01 = w01 & 0x7fff7fffu, m23 = w23 & 0x7fff7fffu;
+    // second-smallest of the four magnitudes, in both halves of t2
+    const uint32_t lo = __vminu2(m01, m23), hi = __vmaxu2(m01, m23);
+    const uint32_t lmax = __vmaxu2(lo, __byte_perm(lo, 0, 0x1032));
+    const uint32_t hmin = __vminu2(hi, __byte_perm(hi, 0, 0x1032));
+    const uint32_t t2 = __vminu2(lmax, hmin);
+    const uint32_t tb = t2 << 16;                       // fp32 bits of t
+    const float t = __uint_as_float(tb);
+    const uint32_t ab[4] = {w01 << 16, w01 & 0xffff0000u, w23 << 16, w23 & 0xffff0000u};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        a[i] = sste_bf16_bits_to_f32(bits[i]);
-        m[i] = fabsf(a[i]);
-        key[i] = ((bits[i] & 0x7fffu) << 2) | static_cast<uint32_t>(3 - i);   // magnitude desc, index asc
-    }
-    // second-smallest magnitude without a sort
-    const float lo1 = fminf(m[0], m[1]), hi1 = fmaxf(m[0], m[1]);
-    const float lo2 = fminf(m[2], m[3]), hi2 = fmaxf(m[2], m[3]);
-    const float t = fminf(fmaxf(lo1, lo2), fminf(hi1, hi2));
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float d = __fsub_rn(m[i], t);
-        float w = __fmul_rn(copysignf(d, a[i]), beta);
+        const float a = __uint_as_float(ab[i]);
+        const float st = __uint_as_float(tb | (ab[i] & 0x80000000u));     // copysign(t, a)
+        float w = __fmul_rn(__fsub_rn(a, st), beta);                        // sign(a) (|a| - t) beta
         if (FP8) w = __fmul_rn(w, wscale);
-        r.w[i] = (d > 0.0f) ? w : 0.0f;
+        r.w[i] = (fabsf(a) > t) ? w : 0.0f;
     }
-    // the two largest keys are kept (keys are pairwise distinct)
-    uint32_t keep = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        int above = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) above += (key[j] > key[i]) ? 1 : 0;
-        keep |= (above < 2 ? 1u : 0u) << i;
-    }
-    r.p0 = __ffs(keep) - 1;
-    r.p1 = 31 - __clz(keep);
+    const uint32_t k0 = (m01 & 0xffffu) * 4u + 3u, k1 = (m01 >> 16) * 4u + 2u;
+    const uint32_t k2 = (m23 & 0xffffu) * 4u + 1u, k3 = (m23 >> 16) * 4u;
+    const uint32_t a = max(k0, k1), b = min(k0, k1), c = max(k2, k3), d = min(k2, k3);
+    const uint32_t top1 = max(a, c), top2 = max(min(a, c), max(b, d));
+    const uint32_t i1 = (top1 & 3u) ^ 3u, i2 = (top2 & 3u) ^ 3u;
+    r.p0 = min(i1, i2);
+    r.p1 = max(i1, i2);
     return r;
-}
-
-__device__ __forceinline__ float sel4(uint32_t idx, float v0, float v1, float v2, float v3)
-{
-    return idx == 0 ? v0 : idx == 1 ? v1 : idx == 2 ? v2 : v3;
 }
 
 // ---------------------------------------------------------------- project + compress
@@ -93,26 +87,24 @@ project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restr
         const int c = i * EW_THREADS + tid;
         const int row = c >> 4, kc = c & 15;
         const uint32_t raw[4] = {in[i].x, in[i].y, in[i].z, in[i].w};
-        uint32_t kept[2][2];   // [group][slot] output bit patterns
-        uint32_t dn[8];        // dense output bit patterns
+        uint32_t kept[2];      // per group: the two kept values, packed (bf16: 32 bits, fp8: 16 bits)
+        uint32_t dn[2][2];     // per group: the four projected values, packed (bf16: two words, fp8: word 0)
         uint32_t mbyte = 0;
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
-            const uint32_t bits[4] = {raw[2 * g] & 0xffffu, raw[2 * g] >> 16, raw[2 * g + 1] & 0xffffu,
-                                      raw[2 * g + 1] >> 16};
-            const SoftGroup s = soft_group<FP8>(bits, beta, wscale);
-            const float v0 = sel4(s.p0, s.w[0], s.w[1], s.w[2], s.w[3]);
-            const float v1 = sel4(s.p1, s.w[0], s.w[1], s.w[2], s.w[3]);
+            const SoftGroup s = soft_group<FP8>(raw[2 * g], raw[2 * g + 1], beta, wscale);
             if (FP8) {
-                kept[g][0] = sste_f32_to_e4m3(v0);
-                kept[g][1] = sste_f32_to_e4m3(v1);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) dn[4 * g + e] = sste_f32_to_e4m3(s.w[e]);
+                const uint32_t e01 = __nv_cvt_float2_to_fp8x2(make_float2(s.w[0], s.w[1]), __NV_SATFINITE, __NV_E4M3);
+                const uint32_t e23 = __nv_cvt_float2_to_fp8x2(make_float2(s.w[2], s.w[3]), __NV_SATFINITE, __NV_E4M3);
+                dn[g][0] = e01 | (e23 << 16);
+                kept[g] = __byte_perm(dn[g][0], 0, s.p0 | (s.p1 << 4) | 0x4400u);
             } else {
-                kept[g][0] = sste_f32_to_bf16_bits(v0);
-                kept[g][1] = sste_f32_to_bf16_bits(v1);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) dn[4 * g + e] = sste_f32_to_bf16_bits(s.w[e]);
+                const __nv_bfloat162 d01 = __floats2bfloat162_rn(s.w[0], s.w[1]);
+                const __nv_bfloat162 d23 = __floats2bfloat162_rn(s.w[2], s.w[3]);
+                dn[g][0] = *reinterpret_cast<const uint32_t *>(&d01);
+                dn[g][1] = *reinterpret_cast<const uint32_t *>(&d23);
+                // halfword p0 -> low half, halfword p1 -> high half
+                kept[g] = __byte_perm(dn[g][0], dn[g][1], 0x1010u + 0x22u * s.p0 + 0x2200u * s.p1);
             }
             mbyte |= (s.p0 | (s.p1 << 2)) << (4 * g);
         }
@@ -123,27 +115,11 @@ project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restr
         const size_t grow = static_cast<size_t>(rb) * PC_ROWS + row;
         const size_t chunk = grow * row_chunks + kb * 16 + kc;   // index in units of 8 input features
         if (FP8) {
-            reinterpret_cast<uint32_t *>(vals)[chunk] =
-                kept[0][0] | (kept[0][1] << 8) | (kept[1][0] << 16) | (kept[1][1] << 24);
-            if (dense) {
-                uint2 d;
-                d.x = dn[0] | (dn[1] << 8) | (dn[2] << 16) | (dn[3] << 24);
-                d.y = dn[4] | (dn[5] << 8) | (dn[6] << 16) | (dn[7] << 24);
-                reinterpret_cast<uint2 *>(dense)[chunk] = d;
-            }
+            reinterpret_cast<uint32_t *>(vals)[chunk] = kept[0] | (kept[1] << 16);
+            if (dense) reinterpret_cast<uint2 *>(dense)[chunk] = make_uint2(dn[0][0], dn[1][0]);
         } else {
-            uint2 v;
-            v.x = kept[0][0] | (kept[0][1] << 16);
-            v.y = kept[1][0] | (kept[1][1] << 16);
-            reinterpret_cast<uint2 *>(vals)[chunk] = v;
-            if (dense) {
-                uint4 d;
-                d.x = dn[0] | (dn[1] << 16);
-                d.y = dn[2] | (dn[3] << 16);
-                d.z = dn[4] | (dn[5] << 16);
-                d.w = dn[6] | (dn[7] << 16);
-                reinterpret_cast<uint4 *>(dense)[chunk] = d;
-            }
+            reinterpret_cast<uint2 *>(vals)[chunk] = make_uint2(kept[0], kept[1]);
+            if (dense) reinterpret_cast<uint4 *>(dense)[chunk] = make_uint4(dn[0][0], dn[0][1], dn[1][0], dn[1][1]);
         }
     }
     __syncthreads();
