@@ -381,15 +381,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     if (PROBE_MODE(p) == 3 && it >= static_cast<uint32_t>(NS)) continue;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, p.status, abort_flag)) { ok = false; break; }
                     const uint32_t lead_full = map_to_cta(full_bar(s), 0);
-                    if (PROBE_MODE(p) == 1 && it >= static_cast<uint32_t>(NS)) {
+                    if ((PROBE_MODE(p) == 1 || PROBE_MODE(p) == 7) && it >= static_cast<uint32_t>(NS)) {
                         if (leader) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full_bar(s)) : "memory");
                         continue;
                     }
-                    if (leader) mbar_arrive_expect_tx(full_bar(s), STAGE_TX);
+                    const bool skip_a = (PROBE_MODE(p) == 4 && it >= static_cast<uint32_t>(NS));   // timing probes:
+                    const bool skip_b = (PROBE_MODE(p) == 5 && it >= static_cast<uint32_t>(NS));   // stale operands
+                    if (leader)
+                        mbar_arrive_expect_tx(full_bar(s), skip_a ? 2u * C::B_STAGE : skip_b ? 2u * C::A_STAGE : STAGE_TX);
                     const uint32_t a_dst = smem_base + s * C::STAGE;
                     const uint32_t b_dst = a_dst + C::A_STAGE;
                     // A: 128 bytes per row = BK/2 compressed (sparse) or BK dense elements
-                    tma_load_2d(a_dst, &map_a, lead_full, kb * (SPARSE ? BK / 2 : BK), m0);
+                    if (!skip_a) tma_load_2d(a_dst, &map_a, lead_full, kb * (SPARSE ? BK / 2 : BK), m0);
+                    if (skip_b) continue;
                     if (BMAJ == BMajor::K) {
 #pragma unroll
                         for (int u = 0; u < B_SUBS; ++u)
@@ -425,7 +429,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         // written by the metadata warps of both CTAs
                         const int atom0 = kb * ATOMS_PER_STAGE;
                         const uint32_t region = group_it % META_REGIONS;
-                        if ((atom0 & 3) == 0 &&
+                        if ((atom0 & 3) == 0 && !(PROBE_MODE(p) >= 6 && group_it >= META_REGIONS) &&
                             !mbar_wait(meta_full_bar(region), (group_it / META_REGIONS) & 1u, p.status, abort_flag)) {
                             ok = false;
                             break;
@@ -646,39 +650,58 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // ------------------------------------------------------------ metadata warps (6..9, both CTAs)
         // HBM -> registers -> tensor memory: lane L of an atom's image is exactly the 16 bytes the
         // instruction expects in tensor-memory lane L, four 32-bit columns per atom.
+        // The loads run three groups (of four atoms) ahead of the stores, in registers: a group's round trip
+        // to L2 / HBM is then off the path that feeds the MMA warp (with load -> store -> signal in sequence
+        // per group, that latency, not the tensor pipe, set the pace of every sparse product).
         const int quarter = warp & 3;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + C::META_COL0;
-        uint32_t group_it = 0;
-        bool ok = true;
-        for (int unit = pair; unit < num_units && ok; unit += num_pairs) {
-            const Unit u = decode(unit);
-            const int tile = u.tile, k_blocks = u.k_blocks;
-            const int mt = tile % m_tiles;
-            const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;
-            const bool rows_valid = m0 < p.M;
-            const uint4 *src = reinterpret_cast<const uint4 *>(meta + static_cast<size_t>(m0 / BM) * k_atoms * 2048) +
-                               quarter * 32 + lane;
-            const int atom_begin = u.split * k_blocks * ATOMS_PER_STAGE;
-            const int atom_end = atom_begin + k_blocks * ATOMS_PER_STAGE;
-            for (int a0 = atom_begin; a0 < atom_end; a0 += 4, ++group_it) {
-                const uint32_t region = group_it % META_REGIONS;
-                if (!mbar_wait_warp(meta_empty_bar(region), ((group_it / META_REGIONS) & 1u) ^ 1u, p.status, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                tc_fence_after();
-                uint4 v[4];
+        // loader cursor: (unit, first atom of the next group)
+        int l_unit = pair, l_a0 = 0, l_end = 0;
+        const uint4 *l_src = nullptr;
+        bool l_rows = false;
+        auto l_setup = [&]() {
+            if (l_unit >= num_units) return;
+            const Unit u = decode(l_unit);
+            const int m0 = (u.tile % m_tiles) * 2 * BM + static_cast<int>(rank) * BM;
+            l_rows = m0 < p.M;
+            l_src = reinterpret_cast<const uint4 *>(meta + static_cast<size_t>(m0 / BM) * k_atoms * 2048) + quarter * 32 + lane;
+            l_a0 = u.split * u.k_blocks * ATOMS_PER_STAGE;
+            l_end = l_a0 + u.k_blocks * ATOMS_PER_STAGE;
+        };
+        auto l_issue = [&](uint4 (&v)[4]) -> bool {
+            if (l_unit >= num_units) return false;
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    v[i] = (rows_valid && a0 + i < k_atoms) ? __ldg(src + static_cast<size_t>(a0 + i) * 128)
-                                                            : make_uint4(0, 0, 0, 0);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) tmem_st_32x4(lane_base + 16 * region + 4 * i, v[i]);
-                tmem_st_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(meta_full_bar(region), 0));
+            for (int i = 0; i < 4; ++i)
+                v[i] = (l_rows && l_a0 + i < k_atoms) ? __ldg(l_src + static_cast<size_t>(l_a0 + i) * 128)
+                                                      : make_uint4(0, 0, 0, 0);
+            l_a0 += 4;
+            if (l_a0 >= l_end) {
+                l_unit += num_pairs;
+                l_setup();
             }
+            return true;
+        };
+        l_setup();
+        uint4 q0[4], q1[4], q2[4];
+        bool h0 = l_issue(q0), h1 = l_issue(q1), h2 = l_issue(q2);
+        uint32_t group_it = 0;
+        while (h0) {
+            if (PROBE_MODE(p) >= 6 && group_it >= META_REGIONS) break;   // timing probe: metadata stays as first written
+            const uint32_t region = group_it % META_REGIONS;
+            if (!mbar_wait_warp(meta_empty_bar(region), ((group_it / META_REGIONS) & 1u) ^ 1u, p.status, abort_flag)) break;
+            tc_fence_after();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) tmem_st_32x4(lane_base + 16 * region + 4 * i, q0[i]);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(meta_full_bar(region), 0));
+            ++group_it;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { q0[i] = q1[i]; q1[i] = q2[i]; }
+            h0 = h1;
+            h1 = h2;
+            h2 = l_issue(q2);
         }
     }
 
