@@ -221,3 +221,31 @@ def linear_bwd_weight(gvals, gmeta, gdt, X, xdt, inv_scale=1.0):
 def linear_bwd_input(dY, gdt, Wt_dense, wdt, inv_scale=1.0):
     """grad_X = grad_Z S(W): [T, O] x [O, I] in fp64 (dense: the 2:4 structure lies along I)."""
     return (decode(dY, gdt) @ decode(Wt_dense, wdt)) * inv_scale
+
+
+# ---------------------------------------------------------------- flip rate (Sec. 3.1, "Flip rate")
+
+def hard_mask(W):
+    """m_h(W): 1 where an element is one of the two largest magnitudes of its group of four.
+
+    Ties are broken as everywhere in this oracle: magnitude descending, then index ascending.
+    W: bf16 bit patterns [rows, k].  Returns uint8 [rows, k].
+    """
+    mag = (np.asarray(W, dtype=np.uint16) & 0x7FFF).astype(np.int64)      # bf16 magnitudes order like integers
+    rows, k = mag.shape
+    g = mag.reshape(rows, k // 4, 4)
+    # stable sort of -magnitude keeps the lower index first among equals
+    order = np.argsort(-g, axis=-1, kind="stable")
+    mask = np.zeros_like(g, dtype=np.uint8)
+    np.put_along_axis(mask, order[..., :2], 1, axis=-1)
+    return mask.reshape(rows, k)
+
+
+def flip_count(W_prev, W_cur):
+    """|| m_h(W_cur) xor m_h(W_prev) ||_1 : the number of mask entries that changed between two iterations."""
+    return int(np.count_nonzero(hard_mask(W_prev) != hard_mask(W_cur)))
+
+
+def flip_rate(W_prev, W_cur):
+    """r_k = || m_h(w_k) xor m_h(w_{k-1}) ||_1 / d  (Sec. 3.1)."""
+    return flip_count(W_prev, W_cur) / float(np.asarray(W_cur).size)
