@@ -205,6 +205,19 @@ sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n, const floa
 /* *out_dev = fl32(fl32(a * b)) for two device scalars (e.g. the product of two inverse scales). */
 sste_status sste_scalar_mul(sste_ctx *ctx, const float *a_dev, const float *b_dev, float *out_dev, void *stream);
 
+/* ---- training diagnostics ---- */
+
+/*
+ * Flip count between two iterations (Sec. 3.1, "Flip rate": r_k = || m_h(w_k) xor m_h(w_{k-1}) ||_1 / d).
+ * meta_prev, meta_cur: device, the metadata images sste_project_compress wrote for the same [rows, k] weight
+ * at two iterations (same dtype, hence same layout; 16-byte aligned).  The 2:4 metadata IS the hard-threshold
+ * mask m_h: the kept pair of a group is its two largest magnitudes.  *count_dev (device, 8-byte aligned)
+ * receives the number of mask entries that differ; the call first sets it to 0 on the stream.  The flip rate
+ * is *count_dev / (rows * k).  Errors: SSTE_ERR_SHAPE unless rows and k are multiples of 128.
+ */
+sste_status sste_flip_count(sste_ctx *ctx, const void *meta_prev, const void *meta_cur, int rows, int k,
+                            unsigned long long *count_dev, void *stream);
+
 /* ---- test / debug helpers ---- */
 
 /* Operand-image metadata -> canonical uint16 [rows, k/16] (see top).  dt selects the 16-bit or 8-bit image. */

@@ -27,7 +27,7 @@ EXPORTS = [
     "sste_vals_bytes", "sste_meta_bytes", "sste_beta_init", "sste_project_compress", "sste_linear_fwd",
     "sste_mvue_sparsify", "sste_linear_bwd_input", "sste_linear_bwd_weight", "sste_amax", "sste_fp8_scale",
     "sste_quantize_fp8", "sste_scalar_mul", "sste_meta_to_canonical", "sste_debug_force_tile_width", "sste_debug_force_splits",
-    "sste_workspace_bytes_recommended", "sste_beta_init_static", "sste_debug_launch_count",
+    "sste_workspace_bytes_recommended", "sste_beta_init_static", "sste_debug_launch_count", "sste_flip_count",
 ]
 
 
@@ -174,6 +174,13 @@ class Context:
 
     def scalar_mul(self, a_dev, b_dev, out_dev):
         self._check(self.lib.sste_scalar_mul(self.handle, _ptr(a_dev), _ptr(b_dev), _ptr(out_dev), _stream()))
+
+    # ---- diagnostics ----------------------------------------------------------------------------
+
+    def flip_count(self, meta_prev, meta_cur, rows, k, count_dev):
+        """sste_flip_count: mask entries that changed between two metadata images of a [rows, k] weight."""
+        self._check(self.lib.sste_flip_count(self.handle, _ptr(meta_prev), _ptr(meta_cur), rows, k, _ptr(count_dev),
+                                             _stream()))
 
     # ---- helpers --------------------------------------------------------------------------------
 

@@ -514,6 +514,37 @@ sste_status launch_result()
     return SSTE_OK;
 }
 
+// ---------------------------------------------------------------- flip count (Sec. 3.1, "Flip rate")
+
+// Number of entries in which the 2:4 masks of two operand images differ.  Both images have the same layout,
+// so nibbles are compared in place: a nibble p0 | p1 << 2 stands for the mask (1 << p0) | (1 << p1).
+__global__ void __launch_bounds__(EW_THREADS)
+flip_count_kernel(const uint4 *__restrict__ a, const uint4 *__restrict__ b, size_t n_vec,
+                  unsigned long long *__restrict__ count)
+{
+    sste_pdl_trigger();
+    sste_pdl_wait();
+    unsigned int local = 0;
+    for (size_t v = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; v < n_vec;
+         v += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const uint4 x = __ldg(a + v), y = __ldg(b + v);
+        const uint32_t wx[4] = {x.x, x.y, x.z, x.w}, wy[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            if (wx[w] == wy[w]) continue;
+#pragma unroll
+            for (int n = 0; n < 8; ++n) {
+                const uint32_t nx = (wx[w] >> (4 * n)) & 0xfu, ny = (wy[w] >> (4 * n)) & 0xfu;
+                const uint32_t mx = (1u << (nx & 3u)) | (1u << (nx >> 2)), my = (1u << (ny & 3u)) | (1u << (ny >> 2));
+                local += __popc(mx ^ my);
+            }
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) local += __shfl_xor_sync(0xffffffffu, local, off);
+    if ((threadIdx.x & 31) == 0 && local) atomicAdd(count, static_cast<unsigned long long>(local));
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------- entry points
@@ -661,5 +692,21 @@ extern "C" sste_status sste_meta_to_canonical(sste_ctx *ctx, const void *meta, i
     else
         sste_launch(meta_to_canonical_kernel<true>, dim3(grid), dim3(EW_THREADS), 0, s,
                     static_cast<const uint8_t *>(meta), rows, k, static_cast<uint16_t *>(canonical_out));
+    return launch_result();
+}
+
+extern "C" sste_status sste_flip_count(sste_ctx *ctx, const void *meta_prev, const void *meta_cur, int rows, int k,
+                                       unsigned long long *count_dev, void *stream)
+{
+    if (!ctx || !meta_prev || !meta_cur || !count_dev) return SSTE_ERR_INVALID_ARG;
+    if (!sste_mult128(rows) || !sste_mult128(k)) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(meta_prev, 16) || !sste_aligned(meta_cur, 16) || !sste_aligned(count_dev, 8)) return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const size_t n_vec = sste_meta_bytes(rows, k) / 16;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    SSTE_CUDA_TRY(cudaMemsetAsync(count_dev, 0, sizeof(unsigned long long), s));
+    sste_launch(flip_count_kernel, dim3(grid_for(n_vec, ctx->sm_count)), dim3(EW_THREADS), 0, s,
+                static_cast<const uint4 *>(meta_prev), static_cast<const uint4 *>(meta_cur), n_vec, count_dev);
     return launch_result();
 }

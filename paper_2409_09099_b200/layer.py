@@ -17,11 +17,12 @@ class SsteLinear:
 
     ``fp8=True`` selects the whole-process FP8 variant (Sec. 5.2): E4M3 forward
     operands, E5M2 output gradient, per-tensor scale = fp8_max / amax computed
-    just in time on the device.
+    just in time on the device.  ``track_flips=True`` keeps the previous iteration's
+    metadata and counts the mask entries that changed at every prune (flip rate, Sec. 3.1).
     """
 
     def __init__(self, ctx: B.Context, W: torch.Tensor, T: int, tensor_id: int = 0, seed: int = 0,
-                 fp8: bool = False, out_dtype: torch.dtype = torch.bfloat16):
+                 fp8: bool = False, out_dtype: torch.dtype = torch.bfloat16, track_flips: bool = False):
         assert W.dtype == torch.bfloat16 and W.is_cuda
         self.ctx, self.W, self.T, self.tensor_id, self.seed, self.fp8 = ctx, W, T, tensor_id, seed, fp8
         self.O, self.I = W.shape
@@ -38,6 +39,11 @@ class SsteLinear:
         self.dX = torch.empty((T, I), dtype=out_dtype, device=dev)
         self.dW = torch.empty((O, I), dtype=out_dtype, device=dev)
         self.launches = 0
+        self.track_flips = track_flips
+        if track_flips:
+            self.meta_prev = torch.empty_like(self.meta)
+            self.flips = torch.zeros(1, dtype=torch.int64, device=dev)   # mask entries changed by the last prune
+            self._have_prev = False
         if fp8:
             self.amax = torch.zeros(3, **f32)          # X, w~ (through W and beta), dY
             self.scale = torch.ones(3, **f32)
@@ -59,6 +65,21 @@ class SsteLinear:
     # (1) prune: w~ = beta * S_soft(W), compressed for the sparse products, dense for grad_X
     def prune(self):
         assert self.beta_ready, "call init_beta() in the first iteration"
+        c = self.ctx
+        if self.track_flips:
+            self.meta, self.meta_prev = self.meta_prev, self.meta     # last iteration's image becomes "previous"
+        self._project()
+        if self.track_flips:
+            if self._have_prev:
+                c.flip_count(self.meta_prev, self.meta, self.O, self.I, self.flips)
+                self.launches += 1
+            self._have_prev = True
+
+    def flip_rate(self) -> float:
+        """r_k of the last prune (synchronises); 0 before the second prune."""
+        return float(self.flips.item()) / (self.O * self.I)
+
+    def _project(self):
         c = self.ctx
         if not self.fp8:
             c.project_compress(self.W, self.beta, self.vals, self.meta, self.w_dense)
