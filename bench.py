@@ -42,7 +42,7 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
-def ncu_traffic(cfg_id: int):
+def ncu_traffic(cfg_id: int, section: str = None):
     """DRAM bytes per launch (read + write) of each stage's kernel, from one ncu capture of this workload.
 
     The figures are measurements recorded in profiles/ncu_dram_traffic.json (with the command that produced
@@ -51,7 +51,8 @@ def ncu_traffic(cfg_id: int):
     path = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
     try:
         with open(path) as f:
-            return json.load(f).get(f"config{cfg_id}", {})
+            rec = json.load(f)
+        return (rec.get(section, {}) if section else rec).get(f"config{cfg_id}", {})
     except (OSError, ValueError):
         return {}
 
@@ -378,6 +379,7 @@ def run_gpu(args):
         tot = {k: sum(ms for _, ms in v) for k, v in per_kernel.items()}
         Ls = cfg["layers"]
         traffic = ncu_traffic(cfg_id)
+        alu_pct = ncu_traffic(cfg_id, "alu_pipe_pct")
         rooflines = {}
         for k in KERNELS:
             avg_ms = tot[k] / len(per_kernel[k])
@@ -387,8 +389,16 @@ def run_gpu(args):
                 # peak of the kernel's own dtype: measured bf16 dense x nominal ratios (2:4 sparse x2, fp8 x2)
                 peak = peaks["bf16_tflops"] * (2.0 if sparse else 1.0) * (2.0 if fp8 else 1.0)
                 ach = fl / (avg_ms * 1e-3) / 1e12
+                # compulsory HBM bytes per launch (operands once in, result once out): the floor of a thin product
+                eb = 1 if fp8 else 2
+                byt = sum((L.T * L.I * eb + L.O * L.I * (eb * (0.5 if sparse else 1.0) + (0.125 if sparse else 0.0))
+                           + L.T * L.O * 2) if k == "linear_fwd" else
+                          (L.O * L.T * (eb * 0.5 + 0.125) + L.T * L.I * eb + L.O * L.I * 2) if k == "linear_bwd_weight" else
+                          (L.T * L.O * eb + L.O * L.I * eb + L.T * L.I * 2) for L in Ls) / len(Ls)
                 rooflines[k] = {"kernel": k, "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
                                 "frac": ach / peak, "traffic": traffic.get(k),
+                                "us_per_launch": avg_ms * 1e3, "tensor_floor_us": fl / (peak * 1e12) * 1e6,
+                                "hbm_floor_us": byt / (peaks["hbm_gbs"] * 1e9) * 1e6,
                                 "peak_source": f"{peaks['source']} cuBLAS bf16 dense burst"
                                                + (" x2 (2:4 sparse, nominal ratio)" if sparse else "")
                                                + (" x2 (fp8, nominal ratio)" if fp8 else "")}
@@ -401,6 +411,11 @@ def run_gpu(args):
                 ach = per_elt * elts / (avg_ms * 1e-3) / 1e9
                 rooflines[k] = {"kernel": k, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                 "frac": ach / peaks["hbm_gbs"], "traffic": traffic.get(k),
+                                "us_per_launch": avg_ms * 1e3,
+                                "hbm_floor_us": per_elt * elts / (peaks["hbm_gbs"] * 1e9) * 1e6,
+                                # ncu: share of the half-rate integer/compare pipe while the kernel runs -- these
+                                # kernels are bound by it, not by HBM
+                                "alu_pipe_pct_ncu": alu_pct.get(k),
                                 "peak_source": f"{peaks['source']} copy bandwidth"}
         dom = max(tot, key=tot.get)
         roofline = rooflines[dom]
@@ -411,7 +426,8 @@ def run_gpu(args):
             cpu_base, _ = time_oracle(cfg_id, min(cfg["layers"][0].T, args.ref_tokens), 5, 1)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms_per_step, "ms_per_step_median": statistics.median(step_ms), "ms_per_step_min": min(step_ms),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "fp8" if fp8 else "bf16", "data": "synthetic",
             "config": workload_config(cfg_id, cfg, world),
             # whole step (sparse and dense products, elementwise kernels) against the nominal 2:4 sparse peak

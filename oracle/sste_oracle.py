@@ -249,3 +249,80 @@ def flip_count(W_prev, W_cur):
 def flip_rate(W_prev, W_cur):
     """r_k = || m_h(w_k) xor m_h(w_{k-1}) ||_1 / d  (Sec. 3.1)."""
     return flip_count(W_prev, W_cur) / float(np.asarray(W_cur).size)
+
+
+# ---------------------------------------------------------------- ablation variants of the pruning step
+# (Sec. 4.1 "Choosing optimal threshold", Eq. 2 hard thresholding, Sec. 4.2 "Minimizing MSE", Sec. 3.2 SR-STE)
+
+def _groups_f32(W):
+    f = bf16_to_f32(_c(W, np.uint16))
+    rows, k = f.shape
+    return f.reshape(rows, k // 4, 4)
+
+
+def _kept_pair(mag_bits):
+    """Positions of the two largest magnitudes per group: magnitude descending, index ascending."""
+    order = np.argsort(-mag_bits.astype(np.int64), axis=-1, kind="stable")[..., :2]
+    return np.sort(order, axis=-1)
+
+
+def project_compress_variant(W, beta32, gamma=0.0, hard=False, odt=BF16, wscale=1.0):
+    """The pruning step with the paper's ablation knobs; returns canonical (vals, meta, dense) like project_compress.
+
+    hard=False: soft thresholding (Eq. 4) with the interpolated threshold t = (1 - gamma) |t2| + gamma |t3|,
+    |t2| <= |t3| the second and third smallest magnitudes (Sec. 4.1: any t in [|t2|, |t3|] is feasible, gamma = 0
+    gives t = |t2|, larger gamma moves t towards |t3|); fp32: t = fl(fl(fl(1 - gamma) * |t2|) + fl(gamma * |t3|)).
+    hard=True: hard thresholding (Eq. 2): the two largest magnitudes are kept unchanged, the others are 0.
+    Then * beta (fp32) [* wscale], one cast, compression of the kept pair.
+    """
+    W = _c(W, np.uint16)
+    rows, k = W.shape
+    a = _groups_f32(W)
+    mag = np.abs(a)
+    bits = (W & 0x7FFF).reshape(rows, k // 4, 4)
+    pair = _kept_pair(bits)
+    f32 = np.float32
+    if hard:
+        keep = np.zeros(a.shape, dtype=bool)
+        np.put_along_axis(keep, pair, True, axis=-1)
+        s = np.where(keep, a, f32(0.0))
+    else:
+        srt = np.sort(mag, axis=-1)
+        g = f32(gamma)
+        t = (f32(1.0) - g) * srt[..., 1] + g * srt[..., 2]          # every step a single fp32 operation
+        t = t.astype(f32)[..., None]
+        d = (a - np.copysign(t, a)).astype(f32)                      # sign(a) (|a| - t)
+        s = np.where(mag > t, d, f32(0.0))
+    w = (s * f32(beta32)).astype(f32)
+    if odt != BF16:
+        w = (w * f32(wscale)).astype(f32)
+    w = np.where(s == 0, f32(0.0), w).astype(f32)                    # pruned entries are canonical +0
+    enc = f32_to_bf16 if odt == BF16 else (lambda x: f32_to_fp8(x, odt))
+    dense = enc(w.reshape(rows, k))
+    vals = np.take_along_axis(dense.reshape(rows, k // 4, 4), pair, axis=-1).reshape(rows, k // 2)
+    nib = (pair[..., 0] | (pair[..., 1] << 2)).astype(np.uint16).reshape(rows, k // 16, 4)
+    meta = (nib[..., 0] | (nib[..., 1] << 4) | (nib[..., 2] << 8) | (nib[..., 3] << 12)).astype(np.uint16)
+    return vals, meta, dense
+
+
+def beta_l1(W):
+    """The L1 rescaling the paper argues against (Sec. 4.2): beta = ||w||_1 / ||S_soft(w)||_1, fp64 sums."""
+    a = _groups_f32(W).astype(np.float64)
+    mag = np.abs(a)
+    t = np.sort(mag, axis=-1)[..., 1:2]
+    s = np.maximum(mag - t, 0.0)
+    den = float(s.sum())
+    return (float(mag.sum()) / den) if den > 0 else 1.0
+
+
+def srste_decay(dW, W, lam):
+    """Sparse-refined STE (Sec. 3.2): the gradient of (lambda / 2) ||w (1 - m_h(w))||^2 added to grad_W.
+
+    dW, W: bf16 bit patterns [O, I]; returns bf16 bits of fl32(dW + fl32(lambda * w)) on pruned entries,
+    dW unchanged on kept ones.
+    """
+    f32 = np.float32
+    g, w = bf16_to_f32(_c(dW, np.uint16)), bf16_to_f32(_c(W, np.uint16))
+    pruned = hard_mask(W) == 0
+    out = np.where(pruned, (g + (f32(lam) * w).astype(f32)).astype(f32), g)
+    return f32_to_bf16(out.astype(f32))
