@@ -205,6 +205,38 @@ sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n, const floa
 /* *out_dev = fl32(fl32(a * b)) for two device scalars (e.g. the product of two inverse scales). */
 sste_status sste_scalar_mul(sste_ctx *ctx, const float *a_dev, const float *b_dev, float *out_dev, void *stream);
 
+/* ---- ablation variants of the pruning step (the axes of the paper's ablations; not on the default path) ---- */
+
+typedef enum { SSTE_PRUNE_SOFT = 0, SSTE_PRUNE_HARD = 1 } sste_pruning;
+
+/*
+ * sste_project_compress with the paper's knobs.  SSTE_PRUNE_SOFT: soft thresholding (Eq. 4) with the
+ * interpolated threshold t = (1 - gamma) |t2| + gamma |t3|, |t2| <= |t3| the second and third smallest
+ * magnitudes of the group (Sec. 4.1; gamma in [0, 1], gamma = 0 is the method and runs the same kernel as
+ * sste_project_compress); fp32: t = fl(fl(fl(1 - gamma) |t2|) + fl(gamma |t3|)).  SSTE_PRUNE_HARD: hard
+ * thresholding (Eq. 2): the two largest magnitudes are kept unchanged, gamma is ignored.  Both are then
+ * multiplied by *beta_dev (pass 1.0 for plain hard thresholding) and cast; all other arguments, layouts and
+ * errors as sste_project_compress; SSTE_ERR_INVALID_ARG for an unknown pruning or gamma outside [0, 1].
+ */
+sste_status sste_project_compress_variant(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
+                                          const float *beta_dev, const float *wscale_dev, sste_dtype odt,
+                                          sste_pruning pruning, float gamma, void *vals, void *meta,
+                                          void *dense_out, void *stream);
+
+/* beta = ||w||_1 / ||S_soft(w)||_1: the magnitude-preserving rescaling the method replaces by Eq. 5 (Sec. 4.2,
+ * "Minimizing MSE").  Arguments, reduction order and degenerate case as sste_beta_init. */
+sste_status sste_beta_init_l1(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, float *beta_dev,
+                              void *stream);
+
+/*
+ * Sparse-refined STE (Sec. 3.2): dW += lambda * w on the entries the 2:4 mask prunes, the gradient of
+ * (lambda / 2) ||w (1 - m_h(w))||^2; kept entries are left as they are.  W [O, I] bf16 and dW [O, I] bf16
+ * (updated in place; fp32 add and multiply, one cast), meta: the metadata image of W written by
+ * sste_project_compress[_variant] (meta_dt: the dtype that image was written for, it selects the layout).
+ */
+sste_status sste_srste_decay(sste_ctx *ctx, const void *W, const void *meta, int O, int I, sste_dtype meta_dt,
+                             float lambda, void *dW, void *stream);
+
 /* ---- training diagnostics ---- */
 
 /*

@@ -16,6 +16,7 @@ _HERE = Path(__file__).resolve().parent
 LIB_PATH = _HERE / "libsste.so"
 
 BF16, F32, E4M3, E5M2 = 0, 1, 2, 3
+PRUNE_SOFT, PRUNE_HARD = 0, 1
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_DTYPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_DEGENERATE, \
     ERR_TIMEOUT = range(10)
 
@@ -28,6 +29,7 @@ EXPORTS = [
     "sste_mvue_sparsify", "sste_linear_bwd_input", "sste_linear_bwd_weight", "sste_amax", "sste_fp8_scale",
     "sste_quantize_fp8", "sste_scalar_mul", "sste_meta_to_canonical", "sste_debug_force_tile_width", "sste_debug_force_splits",
     "sste_workspace_bytes_recommended", "sste_beta_init_static", "sste_debug_launch_count", "sste_flip_count",
+    "sste_project_compress_variant", "sste_beta_init_l1", "sste_srste_decay",
 ]
 
 
@@ -174,6 +176,26 @@ class Context:
 
     def scalar_mul(self, a_dev, b_dev, out_dev):
         self._check(self.lib.sste_scalar_mul(self.handle, _ptr(a_dev), _ptr(b_dev), _ptr(out_dev), _stream()))
+
+    # ---- ablation variants of the pruning step ---------------------------------------------------
+
+    def project_compress_variant(self, W, beta_dev, vals, meta, dense_out=None, wscale_dev=None, hard=False,
+                                 gamma=0.0):
+        O, I = W.shape
+        self._check(self.lib.sste_project_compress_variant(
+            self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev), _ptr(wscale_dev), _CODE_OF[vals.dtype],
+            PRUNE_HARD if hard else PRUNE_SOFT, ctypes.c_float(gamma), _ptr(vals), _ptr(meta), _ptr(dense_out),
+            _stream()))
+
+    def beta_init_l1(self, W, beta_dev):
+        O, I = W.shape
+        self._check(self.lib.sste_beta_init_l1(self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev),
+                                               _stream()))
+
+    def srste_decay(self, W, meta, meta_dt, lam, dW):
+        O, I = W.shape
+        self._check(self.lib.sste_srste_decay(self.handle, _ptr(W), _ptr(meta), O, I, meta_dt, ctypes.c_float(lam),
+                                              _ptr(dW), _stream()))
 
     # ---- diagnostics ----------------------------------------------------------------------------
 

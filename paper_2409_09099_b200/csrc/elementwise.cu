@@ -24,8 +24,10 @@ struct SoftGroup {
 // subtraction a - copysign(t, a), and the kept pair is the top two of four integer keys
 // (magnitude << 2 | 3 - index: magnitude descending, index ascending; pairwise distinct) found with a
 // seven-operation min/max network.
-template <bool FP8>
-__device__ __forceinline__ SoftGroup soft_group(uint32_t w01, uint32_t w23, float beta, float wscale)
+// MODE 0: the method's projection (threshold |t2|); MODE 1: interpolated threshold
+// t = (1 - gamma) |t2| + gamma |t3| (Sec. 4.1); MODE 2: hard thresholding (Eq. 2), the kept pair unchanged.
+template <bool FP8, int MODE>
+__device__ __forceinline__ SoftGroup soft_group(uint32_t w01, uint32_t w23, float beta, float wscale, float gamma)
 {
     SoftGroup r;
     const uint32_t m01 = w01 & 0x7fff7fffu, m23 = w23 & 0x7fff7fffu;
@@ -34,16 +36,22 @@ __device__ __forceinline__ SoftGroup soft_group(uint32_t w01, uint32_t w23, floa
     const uint32_t lmax = __vmaxu2(lo, __byte_perm(lo, 0, 0x1032));
     const uint32_t hmin = __vminu2(hi, __byte_perm(hi, 0, 0x1032));
     const uint32_t t2 = __vminu2(lmax, hmin);
-    const uint32_t tb = t2 << 16;                       // fp32 bits of t
+    uint32_t tb = t2 << 16;                             // fp32 bits of t
+    if (MODE == 1) {                                    // third-smallest magnitude: the other of (lmax, hmin)
+        const float t3 = __uint_as_float(__vmaxu2(lmax, hmin) << 16);
+        tb = __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(1.0f, gamma), __uint_as_float(tb)), __fmul_rn(gamma, t3)));
+    }
     const float t = __uint_as_float(tb);
     const uint32_t ab[4] = {w01 << 16, w01 & 0xffff0000u, w23 << 16, w23 & 0xffff0000u};
+    if (MODE != 2) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float a = __uint_as_float(ab[i]);
-        const float st = __uint_as_float(tb | (ab[i] & 0x80000000u));     // copysign(t, a)
-        float w = __fmul_rn(__fsub_rn(a, st), beta);                        // sign(a) (|a| - t) beta
-        if (FP8) w = __fmul_rn(w, wscale);
-        r.w[i] = (fabsf(a) > t) ? w : 0.0f;
+        for (int i = 0; i < 4; ++i) {
+            const float a = __uint_as_float(ab[i]);
+            const float st = __uint_as_float(tb | (ab[i] & 0x80000000u));     // copysign(t, a)
+            float w = __fmul_rn(__fsub_rn(a, st), beta);                        // sign(a) (|a| - t) beta
+            if (FP8) w = __fmul_rn(w, wscale);
+            r.w[i] = (fabsf(a) > t) ? w : 0.0f;
+        }
     }
     const uint32_t k0 = (m01 & 0xffffu) * 4u + 3u, k1 = (m01 >> 16) * 4u + 2u;
     const uint32_t k2 = (m23 & 0xffffu) * 4u + 1u, k3 = (m23 >> 16) * 4u;
@@ -52,6 +60,16 @@ __device__ __forceinline__ SoftGroup soft_group(uint32_t w01, uint32_t w23, floa
     const uint32_t i1 = (top1 & 3u) ^ 3u, i2 = (top2 & 3u) ^ 3u;
     r.p0 = min(i1, i2);
     r.p1 = max(i1, i2);
+    if (MODE == 2) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float a = __uint_as_float(ab[i]);
+            float w = __fmul_rn(a, beta);
+            if (FP8) w = __fmul_rn(w, wscale);
+            const bool kept = (static_cast<uint32_t>(i) == r.p0) || (static_cast<uint32_t>(i) == r.p1);
+            r.w[i] = (kept && fabsf(a) > 0.0f) ? w : 0.0f;      // a kept zero is +0 like every pruned entry
+        }
+    }
     return r;
 }
 
@@ -60,11 +78,11 @@ __device__ __forceinline__ SoftGroup soft_group(uint32_t w01, uint32_t w23, floa
 // One CTA: 32 rows x 128 input features of W (a quarter of a metadata atom, 512 contiguous bytes of its
 // image); a thread handles two chunks of 8 consecutive features.  Small tiles keep even the 2.4 M-element
 // GPT-2 weights spread over several CTAs per SM.
-template <bool FP8>
+template <bool FP8, int MODE>
 __global__ void __launch_bounds__(EW_THREADS)
 project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restrict__ beta_dev,
-                        const float *__restrict__ wscale_dev, void *__restrict__ vals, uint8_t *__restrict__ meta,
-                        void *__restrict__ dense)
+                        const float *__restrict__ wscale_dev, float gamma, void *__restrict__ vals,
+                        uint8_t *__restrict__ meta, void *__restrict__ dense)
 {
     __shared__ __align__(16) uint8_t meta_s[512];
     const int tid = threadIdx.x;
@@ -92,7 +110,7 @@ project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restr
         uint32_t mbyte = 0;
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
-            const SoftGroup s = soft_group<FP8>(raw[2 * g], raw[2 * g + 1], beta, wscale);
+            const SoftGroup s = soft_group<FP8, MODE>(raw[2 * g], raw[2 * g + 1], beta, wscale, gamma);
             if (FP8) {
                 const uint32_t e01 = __nv_cvt_float2_to_fp8x2(make_float2(s.w[0], s.w[1]), __NV_SATFINITE, __NV_E4M3);
                 const uint32_t e23 = __nv_cvt_float2_to_fp8x2(make_float2(s.w[2], s.w[3]), __NV_SATFINITE, __NV_E4M3);
@@ -140,6 +158,9 @@ __device__ __forceinline__ double warp_sum(double v)
 
 // fp64 sums of <w, s> and <s, s>, s = S_soft(w) in exact arithmetic; per-block partials are
 // combined by the last block in a fixed order.
+// L1 = false: beta = <w, S_soft(w)> / ||S_soft(w)||^2 (Eq. 5); L1 = true: ||w||_1 / ||S_soft(w)||_1 (Sec. 4.2,
+// the rescaling the method replaces).
+template <bool L1>
 __global__ void __launch_bounds__(EW_THREADS)
 beta_kernel(const uint4 *__restrict__ W, size_t n_chunks, double *__restrict__ partials,
             unsigned int *__restrict__ counter, float *__restrict__ beta_dev, unsigned int *__restrict__ status)
@@ -169,7 +190,10 @@ beta_kernel(const uint4 *__restrict__ W, size_t n_chunks, double *__restrict__ p
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const double d = m[i] - t;
-                if (d > 0.0) {
+                if (L1) {
+                    num += m[i];
+                    if (d > 0.0) den += d;
+                } else if (d > 0.0) {
                     const double s = copysign(d, a[i]);
                     num += a[i] * s;
                     den += s * s;
@@ -514,6 +538,46 @@ sste_status launch_result()
     return SSTE_OK;
 }
 
+// ---------------------------------------------------------------- SR-STE decay term (Sec. 3.2)
+
+// grad_W += lambda * w on the entries the 2:4 mask prunes: the gradient of (lambda / 2) ||w (1 - m_h(w))||^2.
+// A thread handles 8 consecutive features of a row (two groups: one metadata byte of the operand image).
+template <bool EIGHT_BIT>
+__global__ void __launch_bounds__(EW_THREADS)
+srste_decay_kernel(const uint4 *__restrict__ W, const uint8_t *__restrict__ meta, int I, size_t n_chunks, float lambda,
+                   uint4 *__restrict__ dW)
+{
+    sste_pdl_trigger();
+    sste_pdl_wait();
+    const size_t row_chunks = static_cast<size_t>(I) / 8;
+    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
+         c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const uint32_t row = static_cast<uint32_t>(c / row_chunks), k = static_cast<uint32_t>(c % row_chunks) * 8u;
+        const size_t atom = static_cast<size_t>(row >> 7) * (I / 128) + (k >> 7);
+        const uint32_t byte = __ldg(meta + atom * 2048 + (EIGHT_BIT ? sste_meta_atom_byte8(row & 127u, k & 127u)
+                                                                     : sste_meta_atom_byte16(row & 127u, k & 127u)));
+        const uint4 w = __ldg(W + c);
+        uint4 g = dW[c];
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+        uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+        for (int grp = 0; grp < 2; ++grp) {
+            const uint32_t nib = (byte >> (4 * grp)) & 0xfu;
+            const uint32_t keep = (1u << (nib & 3u)) | (1u << (nib >> 2));
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (keep & (1u << e)) continue;
+                const int word = 2 * grp + (e >> 1), sh = 16 * (e & 1);
+                const float wv = sste_bf16_bits_to_f32((ww[word] >> sh) & 0xffffu);
+                const float gv = sste_bf16_bits_to_f32((gw[word] >> sh) & 0xffffu);
+                const uint32_t out = sste_f32_to_bf16_bits(__fadd_rn(gv, __fmul_rn(lambda, wv)));
+                gw[word] = (gw[word] & ~(0xffffu << sh)) | (out << sh);
+            }
+        }
+        dW[c] = make_uint4(gw[0], gw[1], gw[2], gw[3]);
+    }
+}
+
 // ---------------------------------------------------------------- flip count (Sec. 3.1, "Flip rate")
 
 // Number of entries in which the 2:4 masks of two operand images differ.  Both images have the same layout,
@@ -549,8 +613,9 @@ flip_count_kernel(const uint4 *__restrict__ a, const uint4 *__restrict__ b, size
 
 // ---------------------------------------------------------------- entry points
 
-extern "C" sste_status sste_beta_init(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, float *beta_dev,
-                                      void *stream)
+namespace {
+
+sste_status beta_launch(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, float *beta_dev, void *stream, bool l1)
 {
     if (!ctx || !W || !beta_dev) return SSTE_ERR_INVALID_ARG;
     if (wdt != SSTE_BF16) return SSTE_ERR_DTYPE;
@@ -560,14 +625,20 @@ extern "C" sste_status sste_beta_init(sste_ctx *ctx, const void *W, int O, int I
     if (!guard.ok) return SSTE_ERR_CUDA;
     const size_t n_chunks = static_cast<size_t>(O) * I / 8;
     const int grid = grid_for(n_chunks, ctx->sm_count);
-    sste_launch(beta_kernel, dim3(grid), dim3(EW_THREADS), 0, static_cast<cudaStream_t>(stream),
-                static_cast<const uint4 *>(W), n_chunks, ctx->partials_dev, ctx->counter_dev, beta_dev, ctx->status_dev);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (l1)
+        sste_launch(beta_kernel<true>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(W), n_chunks,
+                    ctx->partials_dev, ctx->counter_dev, beta_dev, ctx->status_dev);
+    else
+        sste_launch(beta_kernel<false>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(W), n_chunks,
+                    ctx->partials_dev, ctx->counter_dev, beta_dev, ctx->status_dev);
     return launch_result();
 }
 
-extern "C" sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
-                                             const float *beta_dev, const float *wscale_dev, sste_dtype odt,
-                                             void *vals, void *meta, void *dense_out, void *stream)
+// mode: 0 = the method's projection, 1 = interpolated threshold, 2 = hard thresholding
+sste_status project_launch(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, const float *beta_dev,
+                           const float *wscale_dev, sste_dtype odt, int mode, float gamma, void *vals, void *meta,
+                           void *dense_out, void *stream)
 {
     if (!ctx || !W || !beta_dev || !vals || !meta) return SSTE_ERR_INVALID_ARG;
     if (wdt != SSTE_BF16 || (odt != SSTE_BF16 && odt != SSTE_E4M3)) return SSTE_ERR_DTYPE;
@@ -580,12 +651,70 @@ extern "C" sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O
     if (!guard.ok) return SSTE_ERR_CUDA;
     const dim3 grid(I / 128, O / PC_ROWS);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (odt == SSTE_E4M3)
-        sste_launch(project_compress_kernel<true>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(W),
-                    I, beta_dev, wscale_dev, vals, static_cast<uint8_t *>(meta), dense_out);
+    const uint4 *w = static_cast<const uint4 *>(W);
+    uint8_t *m = static_cast<uint8_t *>(meta);
+    const bool f8 = (odt == SSTE_E4M3);
+#define SSTE_PC_LAUNCH(F8, MODE)                                                                                   \
+    sste_launch(project_compress_kernel<F8, MODE>, dim3(grid), dim3(EW_THREADS), 0, s, w, I, beta_dev,           \
+                F8 ? wscale_dev : nullptr, gamma, vals, m, dense_out)
+    if (mode == 0) { if (f8) SSTE_PC_LAUNCH(true, 0); else SSTE_PC_LAUNCH(false, 0); }
+    else if (mode == 1) { if (f8) SSTE_PC_LAUNCH(true, 1); else SSTE_PC_LAUNCH(false, 1); }
+    else { if (f8) SSTE_PC_LAUNCH(true, 2); else SSTE_PC_LAUNCH(false, 2); }
+#undef SSTE_PC_LAUNCH
+    return launch_result();
+}
+
+}  // namespace
+
+extern "C" sste_status sste_beta_init(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, float *beta_dev,
+                                      void *stream)
+{
+    return beta_launch(ctx, W, O, I, wdt, beta_dev, stream, false);
+}
+
+extern "C" sste_status sste_beta_init_l1(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, float *beta_dev,
+                                         void *stream)
+{
+    return beta_launch(ctx, W, O, I, wdt, beta_dev, stream, true);
+}
+
+extern "C" sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
+                                             const float *beta_dev, const float *wscale_dev, sste_dtype odt,
+                                             void *vals, void *meta, void *dense_out, void *stream)
+{
+    return project_launch(ctx, W, O, I, wdt, beta_dev, wscale_dev, odt, 0, 0.0f, vals, meta, dense_out, stream);
+}
+
+extern "C" sste_status sste_project_compress_variant(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
+                                                     const float *beta_dev, const float *wscale_dev, sste_dtype odt,
+                                                     sste_pruning pruning, float gamma, void *vals, void *meta,
+                                                     void *dense_out, void *stream)
+{
+    if (pruning != SSTE_PRUNE_SOFT && pruning != SSTE_PRUNE_HARD) return SSTE_ERR_INVALID_ARG;
+    if (!(gamma >= 0.0f && gamma <= 1.0f)) return SSTE_ERR_INVALID_ARG;
+    const int mode = (pruning == SSTE_PRUNE_HARD) ? 2 : (gamma == 0.0f ? 0 : 1);
+    return project_launch(ctx, W, O, I, wdt, beta_dev, wscale_dev, odt, mode, gamma, vals, meta, dense_out, stream);
+}
+
+extern "C" sste_status sste_srste_decay(sste_ctx *ctx, const void *W, const void *meta, int O, int I,
+                                        sste_dtype meta_dt, float lambda, void *dW, void *stream)
+{
+    if (!ctx || !W || !meta || !dW) return SSTE_ERR_INVALID_ARG;
+    if (meta_dt != SSTE_BF16 && meta_dt != SSTE_E4M3 && meta_dt != SSTE_E5M2) return SSTE_ERR_DTYPE;
+    if (!sste_mult128(O) || !sste_mult128(I)) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(W, 16) || !sste_aligned(meta, 16) || !sste_aligned(dW, 16)) return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const size_t n_chunks = static_cast<size_t>(O) * I / 8;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (meta_dt == SSTE_BF16)
+        sste_launch(srste_decay_kernel<false>, dim3(grid_for(n_chunks, ctx->sm_count)), dim3(EW_THREADS), 0, s,
+                    static_cast<const uint4 *>(W), static_cast<const uint8_t *>(meta), I, n_chunks, lambda,
+                    static_cast<uint4 *>(dW));
     else
-        sste_launch(project_compress_kernel<false>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(W),
-                    I, beta_dev, nullptr, vals, static_cast<uint8_t *>(meta), dense_out);
+        sste_launch(srste_decay_kernel<true>, dim3(grid_for(n_chunks, ctx->sm_count)), dim3(EW_THREADS), 0, s,
+                    static_cast<const uint4 *>(W), static_cast<const uint8_t *>(meta), I, n_chunks, lambda,
+                    static_cast<uint4 *>(dW));
     return launch_result();
 }
 
