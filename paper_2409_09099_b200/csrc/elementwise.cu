@@ -257,6 +257,14 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 
 // ---------------------------------------------------------------- MVUE of one group
 
+// a <= b as an integer mask (all ones / zero) in one instruction
+__device__ __forceinline__ int fset_le(float a, float b)
+{
+    int r;
+    asm("set.le.s32.f32 %0, %1, %2;" : "=r"(r) : "f"(a), "f"(b));
+    return r;
+}
+
 struct MvueGroup {
     uint32_t q0, q1;  // kept positions q0 < q1
     float v0, v1;     // their values before the cast
@@ -297,8 +305,8 @@ __device__ __forceinline__ MvueGroup mvue_group(uint32_t p01, uint32_t p23, floa
     const float r1 = __fmul_rn(u, h);
     const float r2 = __fadd_rn(r1, h);
     // number of cumulative sums at or below each point: compares as 0 / -1, one three-input add each
-    const int j1 = -(((c0 <= r1) ? -1 : 0) + ((c1 <= r1) ? -1 : 0) + ((c2 <= r1) ? -1 : 0));
-    const int n2 = -(((c0 <= r2) ? -1 : 0) + ((c1 <= r2) ? -1 : 0) + ((c2 <= r2) ? -1 : 0));
+    const int j1 = -(fset_le(c0, r1) + fset_le(c1, r1) + fset_le(c2, r1));
+    const int n2 = -(fset_le(c0, r2) + fset_le(c1, r2) + fset_le(c2, r2));
     // index pair before ordering: (other, x) when clipped; (j1, j2) otherwise, where a first point in the
     // last element (j1 = 3) gives the pair (2, 3)
     const int ia_c = (rest == 0.0f) ? (e0 ? 1 : 0) : j1;
@@ -406,10 +414,14 @@ mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t 
         const uint32_t other = __shfl_xor_sync(0xffffffffu, nibs, 8);
         if ((tgl & 1) == 0) {
             const uint32_t k = 4u * tgl;
+            // the eight bytes (own nibble | neighbour's nibble << 4) of columns e = 0..7, four at a time:
+            // even columns from the low nibbles of each byte of `nibs`, odd columns from the high ones
+            const uint32_t even = (nibs & 0x0f0f0f0fu) | ((other << 4) & 0xf0f0f0f0u);
+            const uint32_t odd = ((nibs >> 4) & 0x0f0f0f0fu) | (other & 0xf0f0f0f0u);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 const uint32_t jl = jc * 8 + e;
-                const uint32_t byte = ((nibs >> (4 * e)) & 0xfu) | (((other >> (4 * e)) & 0xfu) << 4);
+                const uint32_t byte = ((e & 1) ? odd : even) >> (8 * (e >> 1));
                 meta_s[FP8 ? sste_meta_atom_byte8(jl, k) : sste_meta_atom_byte16(jl, k)] = static_cast<uint8_t>(byte);
             }
         }
