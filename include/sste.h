@@ -194,6 +194,13 @@ sste_status sste_beta_init_static(int device, const void *W, int O, int I, sste_
  * *amax_dev to 0 on the stream, then raises it with an atomic maximum. */
 sste_status sste_amax(sste_ctx *ctx, const void *x, size_t n, sste_dtype dt, float *amax_dev, void *stream);
 
+/* *amax_dev = max |w~| of the bf16 projection w~ = bf16(beta * S_soft(W)) (what sste_project_compress would
+ * write as dense_out with odt = SSTE_BF16), computed from W [O, I] bf16 and *beta_dev without writing w~: the
+ * scale of the E4M3 weight operand needs this maximum before the operand can be cast (Sec. 5.2).  Bit-identical
+ * to sste_amax of that projection.  The call first sets *amax_dev to 0 on the stream. */
+sste_status sste_project_amax(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, const float *beta_dev,
+                              float *amax_dev, void *stream);
+
 /* *scale_dev = fl32(fp8_max(odt) / *amax_dev) (1 if amax is 0); *inv_scale_dev (nullable) = fl32(1 / scale). */
 sste_status sste_fp8_scale(sste_ctx *ctx, const float *amax_dev, sste_dtype odt, float *scale_dev,
                            float *inv_scale_dev, void *stream);

@@ -29,7 +29,7 @@ EXPORTS = [
     "sste_mvue_sparsify", "sste_linear_bwd_input", "sste_linear_bwd_weight", "sste_amax", "sste_fp8_scale",
     "sste_quantize_fp8", "sste_scalar_mul", "sste_meta_to_canonical", "sste_debug_force_tile_width", "sste_debug_force_splits",
     "sste_workspace_bytes_recommended", "sste_beta_init_static", "sste_debug_launch_count", "sste_flip_count",
-    "sste_project_compress_variant", "sste_beta_init_l1", "sste_srste_decay",
+    "sste_project_compress_variant", "sste_beta_init_l1", "sste_srste_decay", "sste_project_amax",
 ]
 
 
@@ -165,6 +165,11 @@ class Context:
     def amax(self, x, amax_dev):
         self._check(self.lib.sste_amax(self.handle, _ptr(x), ctypes.c_size_t(x.numel()), _CODE_OF[x.dtype],
                                        _ptr(amax_dev), _stream()))
+
+    def project_amax(self, W, beta_dev, amax_dev):
+        O, I = W.shape
+        self._check(self.lib.sste_project_amax(self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev),
+                                               _ptr(amax_dev), _stream()))
 
     def fp8_scale(self, amax_dev, odt, scale_dev, inv_scale_dev=None):
         self._check(self.lib.sste_fp8_scale(self.handle, _ptr(amax_dev), odt, _ptr(scale_dev), _ptr(inv_scale_dev),

@@ -468,6 +468,33 @@ amax_kernel(const uint4 *__restrict__ x, size_t n_chunks, float *__restrict__ am
         atomicMax(reinterpret_cast<unsigned int *>(amax_dev), best << 16);   // non-negative floats order as uints
 }
 
+// amax of the bf16 projection w~ = bf16(beta * S_soft(W)) without writing it: rounding to bf16 is monotone,
+// so the maximum of the rounded magnitudes is the rounded maximum of the fp32 ones.
+__global__ void __launch_bounds__(EW_THREADS)
+project_amax_kernel(const uint4 *__restrict__ W, size_t n_chunks, const float *__restrict__ beta_dev,
+                    float *__restrict__ amax_dev)
+{
+    sste_pdl_trigger();
+    sste_pdl_wait();
+    const float beta = *beta_dev;
+    float best = 0.0f;
+    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
+         c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const uint4 v = __ldg(W + c);
+        const uint32_t raw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            const SoftGroup s = soft_group<false, 0>(raw[2 * g], raw[2 * g + 1], beta, 1.0f, 0.0f);
+            best = fmaxf(best, fmaxf(fmaxf(fabsf(s.w[0]), fabsf(s.w[1])), fmaxf(fabsf(s.w[2]), fabsf(s.w[3]))));
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, off));
+    const uint32_t bits = sste_f32_to_bf16_bits(best);
+    if ((threadIdx.x & 31) == 0 && bits != 0)
+        atomicMax(reinterpret_cast<unsigned int *>(amax_dev), bits << 16);   // non-negative floats order as uints
+}
+
 __global__ void fp8_scale_kernel(const float *amax_dev, float fp8_max, float *scale_dev, float *inv_scale_dev)
 {
     sste_pdl_trigger();
@@ -771,6 +798,23 @@ extern "C" sste_status sste_amax(sste_ctx *ctx, const void *x, size_t n, sste_dt
     SSTE_CUDA_TRY(cudaMemsetAsync(amax_dev, 0, sizeof(float), static_cast<cudaStream_t>(stream)));
     sste_launch(amax_kernel, dim3(grid_for(n_chunks, ctx->sm_count)), dim3(EW_THREADS), 0,
                 static_cast<cudaStream_t>(stream), static_cast<const uint4 *>(x), n_chunks, amax_dev);
+    return launch_result();
+}
+
+extern "C" sste_status sste_project_amax(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
+                                         const float *beta_dev, float *amax_dev, void *stream)
+{
+    if (!ctx || !W || !beta_dev || !amax_dev) return SSTE_ERR_INVALID_ARG;
+    if (wdt != SSTE_BF16) return SSTE_ERR_DTYPE;
+    if (!sste_mult128(O) || !sste_mult128(I)) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(W, 16) || !sste_aligned(amax_dev, 4)) return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const size_t n_chunks = static_cast<size_t>(O) * I / 8;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    SSTE_CUDA_TRY(cudaMemsetAsync(amax_dev, 0, sizeof(float), s));
+    sste_launch(project_amax_kernel, dim3(grid_for(n_chunks, ctx->sm_count)), dim3(EW_THREADS), 0, s,
+                static_cast<const uint4 *>(W), n_chunks, beta_dev, amax_dev);
     return launch_result();
 }
 

@@ -53,8 +53,6 @@ class SsteLinear:
             self.inv_gw = torch.ones(1, **f32)
             self.Xq = torch.empty((T, I), dtype=torch.float8_e4m3fn, device=dev)
             self.dYq = torch.empty((T, O), dtype=torch.float8_e5m2, device=dev)
-            self.w_tilde = torch.empty((O, I), dtype=torch.bfloat16, device=dev)
-            self._v16, self._m16 = ctx.alloc_compressed(O, I, B.BF16)
 
     # (0) first iteration only: beta is computed once and then frozen (Sec. 4.2)
     def init_beta(self):
@@ -85,12 +83,11 @@ class SsteLinear:
             c.project_compress(self.W, self.beta, self.vals, self.meta, self.w_dense)
             self.launches += 1
             return
-        # FP8: the scale of w~ needs amax(w~): project once to bf16, take amax, project again to E4M3
-        c.project_compress(self.W, self.beta, self._v16, self._m16, self.w_tilde)
-        c.amax(self.w_tilde, self.amax[1:2])
+        # FP8: the scale of w~ needs amax(w~) first (one read-only pass over W), then the cast to E4M3
+        c.project_amax(self.W, self.beta, self.amax[1:2])
         c.fp8_scale(self.amax[1:2], B.E4M3, self.scale[1:2], self.inv[1:2])
         c.project_compress(self.W, self.beta, self.vals, self.meta, self.w_dense, wscale_dev=self.scale[1:2])
-        self.launches += 4
+        self.launches += 3
 
     # (2a) forward with the sparse weight
     def forward(self, X):

@@ -173,3 +173,26 @@ def test_fp8_layer_end_to_end(ctx):
     assert rel_fro(Y.float().cpu().numpy(), Y_ref) <= FP8_GEMM_TOL
     assert rel_fro(dW.float().cpu().numpy(), dW_ref) <= FP8_GEMM_TOL
     assert rel_fro(dX.float().cpu().numpy(), dX_ref) <= FP8_GEMM_TOL
+
+
+@pytest.mark.parametrize("O,I", [(128, 128), (384, 640), (1024, 4096)])
+def test_project_amax_equals_amax_of_the_projection(ctx, O, I):
+    """The read-only pass gives bit for bit the amax of the bf16 projection (oracle and GPU two-pass route)."""
+    from paper_2409_09099_b200 import binding as B
+    W = synth.gaussian_bf16(O * 3 + I, (O, I), 0.02)
+    W[0, :4] = orc.f32_to_bf16(np.array([3.0, -2.5, 0.5, 0.25], dtype=np.float32))     # a clear maximum: (3 - 0.5) beta
+    beta32 = np.float32(1.4837)
+    beta = torch.full((1,), float(beta32), dtype=torch.float32, device=DEV)
+    a1 = torch.full((1,), -1.0, dtype=torch.float32, device=DEV)
+    for _ in range(2):                                           # the call zeroes its own accumulator
+        ctx.project_amax(dbf16(W), beta, a1)
+    vals, meta = ctx.alloc_compressed(O, I)
+    dense = torch.empty((O, I), dtype=torch.bfloat16, device=DEV)
+    ctx.project_compress(dbf16(W), beta, vals, meta, dense)
+    a2 = torch.zeros(1, dtype=torch.float32, device=DEV)
+    ctx.amax(dense, a2)
+    ref = orc.amax(orc.project_compress(W, beta32)[2])
+    assert a1.item() == a2.item() == float(ref)
+    zero = torch.zeros((128, 128), dtype=torch.bfloat16, device=DEV)
+    ctx.project_amax(zero, beta, a1)
+    assert a1.item() == 0.0
