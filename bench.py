@@ -178,7 +178,8 @@ def workload_config(cfg_id, cfg, n_gpus):
     return {"workload": f"BASELINE config {cfg_id}: " + ", ".join(f"{L.name} W[{L.O},{L.I}] x {L.T} tokens" for L in cfg["layers"]),
             "precision": "fp8 (e4m3 fwd / e5m2 bwd)" if cfg["fp8"] else "bf16",
             "tokens_per_gpu": cfg["layers"][0].T, "parallelism": f"dp{n_gpus} (token shards; grad_W all-reduced over NCCL when n_gpus > 1)",
-            "l2": "flushed between timed steps (512 MiB write)", "launch": "one CUDA-graph replay per step"}
+            "l2": "flushed between timed steps (512 MiB write)", "launch": "n_gpus = 1: one CUDA-graph replay per step, grad_W on a side stream beside grad_X "
+                      "(--no-overlap, --no-graph switch these off); n_gpus > 1: eager launches"}
 
 
 # --------------------------------------------------------------------------------------------- GPU arm
@@ -227,14 +228,23 @@ def run_gpu(args):
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
-    def layer_step(li, step_idx, mark=lambda: None):
+    overlap = not args.no_overlap and world == 1
+    if overlap:
+        ctx_side = B.Context(local_rank)
+        side_stream = torch.cuda.Stream()
+
+    def layer_step(li, step_idx, mark=lambda: None, serial=False):
         """The five calls of the path for one layer (+ the data-parallel exchange of its grad_W)."""
         lin, X, dY = layers[li]
         mark(); lin.prune()
         mark(); lin.forward(X)
         mark(); lin.sparsify_grad(dY, step_idx, token_offset)
-        mark(); lin.grad_weight()
-        mark(); lin.grad_input(dY)
+        if overlap and not serial:
+            mark(); mark()
+            lin.grad_weight_and_input(dY, ctx_side, side_stream)
+        else:
+            mark(); lin.grad_weight()
+            mark(); lin.grad_input(dY)
         mark()
         # data parallel: the per-rank partial grad_W is summed over ranks (the path's one exchange step)
         return dp.allreduce_grad_w([lin.dW])
@@ -248,7 +258,7 @@ def run_gpu(args):
                 events.append(e)
         handles = []
         for li in range(len(layers)):
-            handles += layer_step(li, step_idx, mark)
+            handles += layer_step(li, step_idx, mark, serial=events is not None)
         for h in handles:
             h.wait()
 
@@ -456,6 +466,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="BASELINE config id (2 = GPT-2-small MLP, the default workload)")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="run grad_W and grad_X back to back instead of grad_W on a side stream beside grad_X")
     ap.add_argument("--no-graph", action="store_true", help="launch the timed steps eagerly instead of replaying a CUDA graph")
     ap.add_argument("--ref-tokens", type=int, default=8192, help="tokens per layer in the CPU-oracle sample")
     args = ap.parse_args()

@@ -112,6 +112,22 @@ class SsteLinear:
         self.grad_input(dY)
         return self.dX, self.dW
 
+    def grad_weight_and_input(self, dY, side_ctx: B.Context, side_stream: torch.cuda.Stream):
+        """grad_W on `side_stream` (through `side_ctx`: its own split-K workspace) while grad_X runs on the
+        current stream: the two products are independent once MVUE has run, and the tail, second split-K pass
+        and ramp-up of one overlap the other.  Both are complete in current-stream order on return."""
+        main = torch.cuda.current_stream()
+        side_stream.wait_stream(main)
+        with torch.cuda.stream(side_stream):
+            saved, self.ctx = self.ctx, side_ctx
+            try:
+                self.grad_weight()
+            finally:
+                self.ctx = saved
+        self.grad_input(dY)
+        main.wait_stream(side_stream)
+        return self.dX, self.dW
+
     # (2b.1) MVUE(dY^T): 2:4 along tokens, compressed and transposed for the grad_W product
     def sparsify_grad(self, dY, step: int = 0, token_offset: int = 0):
         c = self.ctx

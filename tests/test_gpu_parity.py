@@ -264,3 +264,32 @@ def test_argument_validation_launches_nothing(ctx):
     assert e.value.code == B.ERR_DTYPE
     assert ctx.lib.sste_beta_init(ctx.handle, None, 128, 128, 0, None, None) == B.ERR_INVALID_ARG
     assert ctx.poll_device_status() == 0
+
+
+@pytest.mark.parametrize("fp8", [False, True])
+def test_overlapped_backward_equals_serial(ctx, fp8):
+    """grad_W on a side stream (own context, own split-K workspace) beside grad_X gives the same bits as the
+    two calls back to back, also when both products split their reduction."""
+    from paper_2409_09099_b200 import binding as B
+    from paper_2409_09099_b200.layer import SsteLinear
+    O, I, T = 768, 3072, 2048
+    W = dbf16(synth.gaussian_bf16(71, (O, I), 0.02))
+    X = dbf16(synth.gaussian_bf16(72, (T, I), 1.0))
+    dY = dbf16(synth.gaussian_bf16(73, (T, O), 1e-2))
+    side_ctx, side = B.Context(0), torch.cuda.Stream()
+    try:
+        lin = SsteLinear(ctx, W, T, tensor_id=1, seed=9, fp8=fp8)
+        lin.init_beta(); lin.prune(); lin.forward(X)
+        lin.backward(dY, step=2)
+        torch.cuda.synchronize()
+        dW0, dX0 = lin.dW.clone(), lin.dX.clone()
+        lin.dW.zero_(); lin.dX.zero_()
+        for _ in range(3):
+            lin.sparsify_grad(dY, 2)
+            lin.grad_weight_and_input(dY, side_ctx, side)
+        torch.cuda.synchronize()
+        assert torch.equal(lin.dW.view(torch.int16), dW0.view(torch.int16))
+        assert torch.equal(lin.dX.view(torch.int16), dX0.view(torch.int16))
+        assert side_ctx.poll_device_status() == 0
+    finally:
+        side_ctx.close()
