@@ -238,11 +238,12 @@ def run_gpu(args):
         lin, X, dY = layers[li]
         mark(); lin.prune()
         mark(); lin.forward(X)
-        mark(); lin.sparsify_grad(dY, step_idx, token_offset)
         if overlap and not serial:
+            mark(); lin.sparsify_grad(dY, step_idx, token_offset)
             mark(); mark()
             lin.grad_weight_and_input(dY, ctx_side, side_stream)
         else:
+            mark(); lin.sparsify_grad(dY, step_idx, token_offset)
             mark(); lin.grad_weight()
             mark(); lin.grad_input(dY)
         mark()
