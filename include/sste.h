@@ -18,6 +18,14 @@
  *     after a call returns.  Scalars beta / scales are DEVICE pointers to one
  *     float so that no call needs a host synchronisation.
  *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it.
+ *     Kernels are launched with programmatic stream serialisation: a kernel of
+ *     this library may be scheduled while the previous kernel of the stream
+ *     drains, but reads or writes global memory only once that kernel has
+ *     completed, so stream order holds for every caller-visible effect, also
+ *     between these calls and the caller's own kernels, copies and captures.
+ *   - Two calls that may overlap on the device (different streams) need
+ *     different contexts if either is a product: the split-K workspace belongs
+ *     to the context.
  *   - O = out features, I = in features, T = tokens.  O, I and T must be
  *     multiples of 128 and tensor pointers 128-byte aligned, otherwise
  *     SSTE_ERR_SHAPE / SSTE_ERR_ALIGN is returned BEFORE anything is launched.
