@@ -112,6 +112,23 @@ class SsteLinear:
         self.grad_input(dY)
         return self.dX, self.dW
 
+    def grad_input_mvue_weight(self, dY, step: int = 0, tensor_id_w: int | None = None):
+        """Ablation (Sec. 5.1, the variant the paper rejects): grad_X = dY MVUE(S(W)^T)^T on sparse tensor cores.
+
+        The sparsified operand must be 2:4 along the contraction dim O, so MVUE runs on w~ viewed as [O, I]
+        (groups of four consecutive rows), giving the compressed [I, O] operand; the product is then the
+        forward-type call with dY as the K-major operand.  bf16 only.  Composed of existing calls.
+        """
+        assert not self.fp8
+        c = self.ctx
+        if not hasattr(self, "wt_vals"):
+            self.wt_vals, self.wt_meta = c.alloc_compressed(self.I, self.O, B.BF16)
+        tid = self.tensor_id + (1 << 16) if tensor_id_w is None else tensor_id_w     # a stream of its own
+        c.mvue_sparsify(self.w_dense, self.seed, tid, step, self.wt_vals, self.wt_meta)
+        c.linear_fwd(dY, self.wt_vals, self.wt_meta, self.dX)
+        self.launches += 2
+        return self.dX
+
     def grad_weight_and_input(self, dY, side_ctx: B.Context, side_stream: torch.cuda.Stream):
         """grad_W on `side_stream` (through `side_ctx`: its own split-K workspace) while grad_X runs on the
         current stream: the two products are independent once MVUE has run, and the tail, second split-K pass

@@ -6,7 +6,7 @@ import torch
 
 from oracle import sste_oracle as orc
 from paper_2409_09099_b200 import synth
-from tests.gpu_util import DEV, bits16, bits8, canonical_meta, dbf16
+from tests.gpu_util import DEV, bits16, bits8, canonical_meta, dbf16, rel_fro
 
 pytestmark = pytest.mark.gpu
 
@@ -94,3 +94,34 @@ def test_srste_decay(ctx, fp8):
     g = dbf16(dW)
     ctx.srste_decay(dbf16(W), meta, dt, lam, g)
     assert np.array_equal(bits16(g), orc.srste_decay(dW, W, lam))
+
+
+def test_grad_input_with_mvue_on_the_weight(ctx):
+    """The rejected ablation of Sec. 5.1 (MVUE on S(W) for grad_X), composed of existing calls: operand bits equal
+    the oracle's MVUE of w~ along O, the product matches fp64, and the estimator is unbiased over steps."""
+    from paper_2409_09099_b200 import binding as B
+    from paper_2409_09099_b200.layer import SsteLinear
+    O, I, T = 256, 384, 512
+    W = synth.gaussian_bf16(31, (O, I), 0.02)
+    X = synth.gaussian_bf16(32, (T, I), 1.0)
+    dY = synth.gaussian_bf16(33, (T, O), 1e-2)
+    lin = SsteLinear(ctx, dbf16(W), T, tensor_id=2, seed=5)
+    lin.init_beta(); lin.prune(); lin.forward(dbf16(X))
+    lin.grad_input_mvue_weight(dbf16(dY), step=4)
+    torch.cuda.synchronize()
+    _, _, wt = orc.project_compress(W, np.float32(lin.beta.item()))
+    ogv, ogm, _, _ = orc.mvue(wt, 5, 2 + (1 << 16), 4)                   # w~ [O, I] sparsified along O -> [I, O]
+    assert np.array_equal(bits16(lin.wt_vals), ogv)
+    assert np.array_equal(canonical_meta(ctx, lin.wt_meta, I, O, B.BF16), ogm)
+    ref = orc.linear_fwd(dY, orc.BF16, ogv, ogm, orc.BF16)               # dX[T, I] = dY MVUE(w~^T)^T
+    assert rel_fro(lin.dX.float().cpu().numpy(), ref) <= 1e-2
+    # unbiased: the mean over steps approaches the dense grad_X (statistical bound: 6 sigma of the sample mean)
+    exact = orc.linear_bwd_input(dY, orc.BF16, wt, orc.BF16)
+    acc = np.zeros_like(exact)
+    n = 64
+    for s in range(n):
+        lin.grad_input_mvue_weight(dbf16(dY), step=100 + s)
+        acc += lin.dX.float().cpu().numpy()
+    err = np.linalg.norm(acc / n - exact) / np.linalg.norm(exact)
+    one = np.linalg.norm(lin.dX.float().cpu().numpy() - exact) / np.linalg.norm(exact)
+    assert err < 6.0 * one / np.sqrt(n) + 5e-3
