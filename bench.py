@@ -381,6 +381,37 @@ def run_gpu(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
     e2e_value = world * flops_step / (e2e_ms * 1e-3) / 1e12
+    # ---- every stage on its own, hot: 10 calls back to back inside one CUDA graph (no launch or event gaps,
+    # operands L2-resident where they fit) -- the kernel-level companion of the per-stage times above
+    hot_us = {}
+    if world == 1:
+        calls = {
+            "project_compress": lambda lin, X, dY: lin.prune(),
+            "linear_fwd": lambda lin, X, dY: lin.forward(X),
+            "mvue_sparsify": lambda lin, X, dY: lin.sparsify_grad(dY, 0, token_offset),
+            "linear_bwd_weight": lambda lin, X, dY: lin.grad_weight(),
+            "linear_bwd_input": lambda lin, X, dY: lin.grad_input(dY),
+        }
+        reps = 10
+        for k, fn in calls.items():
+            per_layer = []
+            for lin, X, dY in layers:
+                fn(lin, X, dY)
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    for _ in range(reps):
+                        fn(lin, X, dY)
+                g.replay()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                g.replay()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                per_layer.append(e0.elapsed_time(e1) / reps * 1e3)
+                del g
+            hot_us[k] = sum(per_layer) / len(per_layer)
     status = ctx.poll_device_status()
 
     if rank == 0:
@@ -408,7 +439,9 @@ def run_gpu(args):
                           (L.T * L.O * eb + L.O * L.I * eb + L.T * L.I * 2) for L in Ls) / len(Ls)
                 rooflines[k] = {"kernel": k, "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
                                 "frac": ach / peak, "traffic": traffic.get(k),
-                                "us_per_launch": avg_ms * 1e3, "tensor_floor_us": fl / (peak * 1e12) * 1e6,
+                                "us_per_launch": avg_ms * 1e3, "us_per_launch_hot": hot_us.get(k),
+                                "frac_hot": (fl / (hot_us[k] * 1e-6) / 1e12 / peak) if k in hot_us else None,
+                                "tensor_floor_us": fl / (peak * 1e12) * 1e6,
                                 "hbm_floor_us": byt / (peaks["hbm_gbs"] * 1e9) * 1e6,
                                 "peak_source": f"{peaks['source']} cuBLAS bf16 dense burst"
                                                + (" x2 (2:4 sparse, nominal ratio)" if sparse else "")
@@ -422,7 +455,9 @@ def run_gpu(args):
                 ach = per_elt * elts / (avg_ms * 1e-3) / 1e9
                 rooflines[k] = {"kernel": k, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                 "frac": ach / peaks["hbm_gbs"], "traffic": traffic.get(k),
-                                "us_per_launch": avg_ms * 1e3,
+                                "us_per_launch": avg_ms * 1e3, "us_per_launch_hot": hot_us.get(k),
+                                "frac_hot": (per_elt * elts / (hot_us[k] * 1e-6) / 1e9 / peaks["hbm_gbs"])
+                                if k in hot_us else None,
                                 "hbm_floor_us": per_elt * elts / (peaks["hbm_gbs"] * 1e9) * 1e6,
                                 # ncu: share of the half-rate integer/compare pipe while the kernel runs -- these
                                 # kernels are bound by it, not by HBM
