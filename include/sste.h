@@ -31,8 +31,10 @@
  *     SSTE_ERR_SHAPE / SSTE_ERR_ALIGN is returned BEFORE anything is launched.
  *   - A device that is not compute capability 10.x gives SSTE_ERR_ARCH.  There
  *     is no CPU or other fallback.
- *   - Kernels never trap.  Bounded waits that expire record SSTE_ERR_TIMEOUT
- *     in the context's device status word, read by sste_poll_device_status.
+ *   - Kernels never trap.  Every device-side wait is bounded (2 s of wall time,
+ *     %globaltimer); one that expires records SSTE_ERR_TIMEOUT in the context's
+ *     device status word, read by sste_poll_device_status, and the kernel leaves
+ *     with that product's output incomplete: poll before trusting results.
  *   - bf16 tensors hold IEEE bfloat16 bit patterns, E4M3 is the "fn" flavour
  *     (max 448, no infinity), E5M2 is IEEE-like (max finite 57344).
  *
@@ -181,7 +183,8 @@ sste_status sste_linear_bwd_weight(sste_ctx *ctx, const void *gvals, const void 
  * no workspace to lend and therefore no sste_ctx.  This call needs neither: its reduction scratch is a
  * fixed array inside the library image (about 129 KB that every GPU loading the library holds until the
  * process exits).  It calls no cudaMalloc / cudaFree or other allocating routine.
- *   device   ordinal of the GPU that W and beta_dev live on (made current for the call).
+ *   device   ordinal of the GPU that W and beta_dev live on (made current for the call); SSTE_ERR_ARCH
+ *            unless it is compute capability 10.x.
  *   W        bf16 [O, I], O and I multiples of 128.  One partial per 128 x 128 tile is kept, and the array
  *            holds 8192 of them: (O/128)*(I/128) > 8192 returns SSTE_ERR_WORKSPACE and launches nothing.
  *   beta_dev device float, written asynchronously on `stream`.  If S_soft(W) is identically zero it

@@ -58,26 +58,15 @@ extern "C" sste_status sste_create(sste_ctx **out, int device, void *workspace, 
     ctx->counter_dev = reinterpret_cast<unsigned int *>(ws + SSTE_WS_COUNTER_OFF);
     ctx->partials_dev = reinterpret_cast<double *>(ws + SSTE_WS_PARTIALS_OFF);
     ctx->cu_tensor_map_encode = encode;
-    ctx->splitk_counters = nullptr;
     ctx->splitk_partials = nullptr;
     ctx->splitk_partial_bytes = 0;
     if (workspace_bytes > SSTE_WS_SPLITK_PARTIALS_OFF + (size_t(1) << 20)) {
-        ctx->splitk_counters = reinterpret_cast<unsigned int *>(ws + SSTE_WS_SPLITK_COUNTERS_OFF);
         ctx->splitk_partials = reinterpret_cast<float *>(ws + SSTE_WS_SPLITK_PARTIALS_OFF);
         ctx->splitk_partial_bytes = workspace_bytes - SSTE_WS_SPLITK_PARTIALS_OFF;
-        if (cudaMemset(ctx->splitk_counters, 0, sizeof(unsigned int) * SSTE_SPLITK_COUNTERS) != cudaSuccess) {
-            delete ctx;
-            return SSTE_ERR_CUDA;
-        }
     }
     if (cudaMemset(ws, 0, SSTE_WS_PARTIALS_OFF) != cudaSuccess) {
         delete ctx;
         return SSTE_ERR_CUDA;
-    }
-    sste_status st = sste_gemm_launch_check(ctx);
-    if (st != SSTE_OK) {
-        delete ctx;
-        return st;
     }
     *out = ctx;
     return SSTE_OK;

@@ -17,7 +17,6 @@ struct sste_ctx {
     unsigned int *counter_dev;  // ticket counter of the beta reduction
     double *partials_dev;       // 2 doubles per reduction block
     void *cu_tensor_map_encode; // cuTensorMapEncodeTiled, resolved through the runtime
-    unsigned int *splitk_counters;  // SSTE_SPLITK_COUNTERS arrival counters (zero between launches)
     float *splitk_partials;         // fp32 partial tiles of split-K products; null if the workspace is minimal
     size_t splitk_partial_bytes;
 };
@@ -28,9 +27,7 @@ constexpr size_t SSTE_WS_COUNTER_OFF = 64;
 constexpr size_t SSTE_WS_PARTIALS_OFF = 256;
 constexpr size_t SSTE_WS_BYTES = SSTE_WS_PARTIALS_OFF + 2 * sizeof(double) * SSTE_MAX_REDUCE_BLOCKS;
 // optional tail of the workspace, used by split-K products
-constexpr int SSTE_SPLITK_COUNTERS = 8192;
-constexpr size_t SSTE_WS_SPLITK_COUNTERS_OFF = (SSTE_WS_BYTES + 255) / 256 * 256;
-constexpr size_t SSTE_WS_SPLITK_PARTIALS_OFF = SSTE_WS_SPLITK_COUNTERS_OFF + sizeof(unsigned int) * SSTE_SPLITK_COUNTERS;
+constexpr size_t SSTE_WS_SPLITK_PARTIALS_OFF = (SSTE_WS_BYTES + 1023) / 1024 * 1024;
 constexpr size_t SSTE_WS_RECOMMENDED_BYTES = SSTE_WS_SPLITK_PARTIALS_OFF + (size_t(192) << 20);
 
 static inline bool sste_mult128(int v) { return v > 0 && (v % 128) == 0; }
@@ -115,6 +112,3 @@ inline cudaError_t sste_launch(void (*kern)(KArgs...), dim3 grid, dim3 block, si
 
 // Process-wide count of kernels this library has launched (read by sste_debug_launch_count).
 void sste_count_launches(int n);
-
-// entry points implemented in the other translation units
-sste_status sste_gemm_launch_check(const sste_ctx *ctx);

@@ -16,6 +16,8 @@
 // Every wait is bounded: on expiry the CTA records SSTE_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace {
@@ -24,7 +26,7 @@ constexpr int BM = 128;            // rows of A per CTA (a pair covers 256)
 constexpr int TMEM_COLS = 512;
 constexpr int META_REGIONS = 8;   // metadata regions of 16 columns (four atoms) after the accumulators
 constexpr int STAGING_BYTES = 32768;   // two epilogue panels of 128 x 64 bf16
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // two seconds of wall time (%globaltimer)
 
 enum class BMajor { K, MN };
 
@@ -78,15 +80,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 // Bounded wait of ONE thread.  Returns false (after recording a timeout) instead of spinning forever.
+// The limit is wall time (nanoseconds of %globaltimer), so it does not depend on the SM clock.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned int *status, volatile int *abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long start = clock64();
+    const unsigned long long start = global_ns();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - start > WAIT_LIMIT_CYCLES) {
+        if (global_ns() - start > WAIT_LIMIT_NS) {
             atomicCAS(status, 0u, static_cast<unsigned int>(SSTE_ERR_TIMEOUT));
             *abort_flag = 1;
             return false;
@@ -126,6 +135,22 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
 __device__ __forceinline__ void epilogue_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier of the 128 epilogue threads that also combines a flag: true only if every thread passed true.
+// The four epilogue warps wait for an accumulator separately; they must leave TOGETHER when one wait
+// expired, or the others would park at the next epilogue barrier for good.
+__device__ __forceinline__ bool epilogue_all(bool ok)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 1, 128, p;\n\t"
+        "selp.b32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"(ok ? 1u : 0u)
+        : "memory");
+    return r != 0;
+}
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
 {
@@ -221,27 +246,7 @@ struct GemmParams {
     int splits;             // split-K factor of the tiles from `split_from` on (1 = none)
     int split_from;         // first split tile: tiles below it are computed whole
     float *partials;        // split-K: fp32 partial tiles [tile][cta][split][128][BN], summed by splitk_reduce_kernel
-#ifdef SSTE_PROBE
-    int probe;              // 1: skip the loads after the first ring fill, 2: skip the MMAs
-    long long *dbg;         // clock64 stamps of pair 0: [tile][0..3] = mma start, mma issued, acc full seen, epilogue done
-#endif
 };
-#ifdef SSTE_PROBE
-int g_probe_mode = 0;
-long long *g_probe_dbg = nullptr;
-#define PROBE_MODE(p) ((p).probe)
-#define PROBE_STAMP(p, tile, k) do { if ((p).dbg && blockIdx.x == 0 && (tile) < 16) (p).dbg[(tile) * 4 + (k)] = clock64(); } while (0)
-// kernel-level stamps: [64 + k] = clock64 of CTA 0, [72 + k] = globaltimer of CTA 0, [80] / [81] = min entry / max exit (ns) over CTAs
-__device__ __forceinline__ long long probe_gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define PROBE_KSTAMP(p, k) do { if ((p).dbg && threadIdx.x == 0) { long long g__ = probe_gtime(); \
-    if (blockIdx.x == 0) { (p).dbg[64 + (k)] = clock64(); (p).dbg[72 + (k)] = g__; } \
-    if ((k) == 0) atomicMin(reinterpret_cast<unsigned long long *>((p).dbg + 80), static_cast<unsigned long long>(g__)); \
-    if ((k) == 2) atomicMax(reinterpret_cast<unsigned long long *>((p).dbg + 81), static_cast<unsigned long long>(g__)); } } while (0)
-#else
-#define PROBE_KSTAMP(p, k) do { } while (0)
-#define PROBE_MODE(p) 0
-#define PROBE_STAMP(p, tile, k) do { } while (0)
-#endif
 
 // 32 lanes x 4 consecutive 32-bit columns <- 4 registers per thread
 __device__ __forceinline__ void tmem_st_32x4(uint32_t taddr, uint4 v)
@@ -281,7 +286,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint8_t *__restrict__ meta, const GemmParams p)
 {
     sste_pdl_trigger();
-    PROBE_KSTAMP(p, 0);
     using C = Cfg<SPARSE, BN>;
     constexpr int NS = C::STAGES;
     constexpr int NB = C::ACC_BUFS;
@@ -360,7 +364,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     cluster_sync();          // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     sste_pdl_wait();         // everything above overlapped the previous kernel; global memory from here on
-    PROBE_KSTAMP(p, 1);
     const uint32_t tmem_base = *tmem_slot_ptr;
 
     if (warp == 0) {
@@ -377,22 +380,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 for (int kb = kb0; kb < kb0 + k_blocks; ++kb, ++it) {
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1u;
-                    if (PROBE_MODE(p) == 3 && it >= static_cast<uint32_t>(NS)) continue;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, p.status, abort_flag)) { ok = false; break; }
                     const uint32_t lead_full = map_to_cta(full_bar(s), 0);
-                    if ((PROBE_MODE(p) == 1 || PROBE_MODE(p) == 7) && it >= static_cast<uint32_t>(NS)) {
-                        if (leader) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full_bar(s)) : "memory");
-                        continue;
-                    }
-                    const bool skip_a = (PROBE_MODE(p) == 4 && it >= static_cast<uint32_t>(NS));   // timing probes:
-                    const bool skip_b = (PROBE_MODE(p) == 5 && it >= static_cast<uint32_t>(NS));   // stale operands
-                    if (leader)
-                        mbar_arrive_expect_tx(full_bar(s), skip_a ? 2u * C::B_STAGE : skip_b ? 2u * C::A_STAGE : STAGE_TX);
+                    if (leader) mbar_arrive_expect_tx(full_bar(s), STAGE_TX);
                     const uint32_t a_dst = smem_base + s * C::STAGE;
                     const uint32_t b_dst = a_dst + C::A_STAGE;
                     // A: 128 bytes per row = BK/2 compressed (sparse) or BK dense elements
-                    if (!skip_a) tma_load_2d(a_dst, &map_a, lead_full, kb * (SPARSE ? BK / 2 : BK), m0);
-                    if (skip_b) continue;
+                    tma_load_2d(a_dst, &map_a, lead_full, kb * (SPARSE ? BK / 2 : BK), m0);
                     if (BMAJ == BMajor::K) {
 #pragma unroll
                         for (int u = 0; u < B_SUBS; ++u)
@@ -417,7 +411,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const uint32_t buf = local_tile % NB, use = local_tile / NB;
                 if (!mbar_wait(acc_empty_bar(buf), (use & 1u) ^ 1u, p.status, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                PROBE_STAMP(p, local_tile, 0);
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {     // stage index inside the unit's K range
                     const int s = it % NS;
@@ -428,21 +421,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         // written by the metadata warps of both CTAs
                         const int atom0 = kb * ATOMS_PER_STAGE;
                         const uint32_t region = group_it % META_REGIONS;
-                        if ((atom0 & 3) == 0 && !(PROBE_MODE(p) >= 6 && group_it >= META_REGIONS) &&
+                        if ((atom0 & 3) == 0 &&
                             !mbar_wait(meta_full_bar(region), (group_it / META_REGIONS) & 1u, p.status, abort_flag)) {
                             ok = false;
                             break;
                         }
                         meta_cols = tmem_base + C::META_COL0 + 16 * region + 4 * (atom0 & 3);
                     }
-                    if (!(PROBE_MODE(p) == 3 && it >= static_cast<uint32_t>(NS)) &&
-                        !mbar_wait(full_bar(s), ph, p.status, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(s), ph, p.status, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_src = smem_base + s * C::STAGE;
                     const uint32_t b_src = a_src + C::A_STAGE;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        if (PROBE_MODE(p) == 2) break;
                         const uint64_t adesc = smem_desc(a_src + 32 * j, 16, 1024, 2);
                         uint64_t bdesc;
                         if (BMAJ == BMajor::K) {
@@ -473,7 +464,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     }
                 }
                 if (ok) tc_commit_pair(acc_full_bar(buf));
-                PROBE_STAMP(p, local_tile, 1);
             }
         }
     } else if (warp < 6) {
@@ -494,9 +484,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint32_t buf = local_tile % NB, use = local_tile / NB;
             const uint32_t acc_base = lane_base + buf * BN;
             const uint32_t lead_acc_empty = map_to_cta(acc_empty_bar(buf), 0);
-            if (!mbar_wait_warp(acc_full_bar(buf), use & 1u, p.status, abort_flag)) { ok = false; break; }
+            if (!epilogue_all(mbar_wait_warp(acc_full_bar(buf), use & 1u, p.status, abort_flag))) { ok = false; break; }
             tc_fence_after();
-            if (threadIdx.x == 64) PROBE_STAMP(p, local_tile, 2);
             if (OUT_F32) {
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -524,10 +513,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 }
                 tc_fence_before();
                 epilogue_barrier();
-                if (store_thread) {
-                    PROBE_STAMP(p, local_tile, 3);
-                    mbar_arrive_cluster(lead_acc_empty);
-                }
+                if (store_thread) mbar_arrive_cluster(lead_acc_empty);
                 continue;
             }
             if (unit >= p.split_from && p.splits > 1) {
@@ -559,10 +545,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 }
                 tc_fence_before();
                 epilogue_barrier();
-                if (store_thread) {
-                    PROBE_STAMP(p, local_tile, 3);
-                    mbar_arrive_cluster(lead_acc_empty);
-                }
+                if (store_thread) mbar_arrive_cluster(lead_acc_empty);
                 continue;
             }
             // bf16 output in panels of 64 columns through two 16 KB staging buffers and TMA stores.
@@ -629,10 +612,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             tc_fence_before();
             {
                 const uint32_t off = acquire_staging();      // includes the barrier after everyone's loads
-                if (store_thread) {
-                    PROBE_STAMP(p, local_tile, 3);
-                    mbar_arrive_cluster(lead_acc_empty);
-                }
+                if (store_thread) mbar_arrive_cluster(lead_acc_empty);
                 stage_chunk(r0, staging_generic + off, 0);
                 stage_chunk(r1, staging_generic + off, 32);
                 store_panel(off, DIRECT_PANELS);
@@ -685,7 +665,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         bool h0 = l_issue(q0), h1 = l_issue(q1), h2 = l_issue(q2);
         uint32_t group_it = 0;
         while (h0) {
-            if (PROBE_MODE(p) >= 6 && group_it >= META_REGIONS) break;   // timing probe: metadata stays as first written
             const uint32_t region = group_it % META_REGIONS;
             if (!mbar_wait_warp(meta_empty_bar(region), ((group_it / META_REGIONS) & 1u) ^ 1u, p.status, abort_flag)) break;
             tc_fence_after();
@@ -712,7 +691,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
-    PROBE_KSTAMP(p, 2);
 }
 
 // ------------------------------------------------------------------ host side
@@ -772,6 +750,21 @@ splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, i
     }
 }
 
+// Runs `fn` once per device ordinal (and again after a failure); thread-safe.
+struct DeviceOnce {
+    static constexpr int MAX_DEVICES = 64;
+    std::mutex mu;
+    bool done[MAX_DEVICES] = {};
+    template <typename F>
+    bool run(int device, F fn)
+    {
+        if (device < 0 || device >= MAX_DEVICES) return fn();
+        std::lock_guard<std::mutex> lock(mu);
+        if (!done[device]) done[device] = fn();
+        return done[device];
+    }
+};
+
 struct SplitPlan { int splits, split_from; };
 SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn);
 
@@ -800,12 +793,13 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
     }
     if (!ok) return SSTE_ERR_CUDA;
     auto kern = gemm_kernel<SPARSE, BMAJ, ELT, BN, OUT_T, OUT_F32>;
-    static bool attr_set = false;   // per instantiation
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
-            return SSTE_ERR_CUDA;
-        attr_set = true;
-    }
+    // The opt-in to more than 48 KB of dynamic shared memory is a per-DEVICE attribute of the kernel:
+    // set once per (instantiation, device), under a lock (contexts may be used from several host threads).
+    static DeviceOnce attr_done;
+    if (!attr_done.run(ctx->device, [&] {
+            return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) == cudaSuccess;
+        }))
+        return SSTE_ERR_CUDA;
     const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM), n_tiles = (p.N + BN - 1) / BN;
     GemmParams pp = p;
     const int tiles = m_tiles * n_tiles;
@@ -817,10 +811,6 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
     const int n_split_tiles = tiles - pp.split_from;
     int pairs = pp.split_from + n_split_tiles * pp.splits;
     if (pairs > ctx->sm_count / 2) pairs = ctx->sm_count / 2;
-#ifdef SSTE_PROBE
-    pp.probe = g_probe_mode;
-    pp.dbg = g_probe_dbg;
-#endif
     map_p = map_a;   // unused without split-K
     if (pp.splits > 1 &&
         !make_map(ctx, &map_p, pp.partials, 4, static_cast<uint64_t>(n_split_tiles) * 2 * pp.splits * BM, BN, 32, BM,
@@ -926,7 +916,6 @@ sste_status launch_out(const sste_ctx *ctx, const void *A, const void *B, const 
 
 }  // namespace
 
-sste_status sste_gemm_launch_check(const sste_ctx *) { return SSTE_OK; }
 extern "C" sste_status sste_debug_force_splits(int splits)
 {
     if (splits < 0 || splits > 4) return SSTE_ERR_INVALID_ARG;
@@ -939,10 +928,6 @@ extern "C" sste_status sste_debug_force_tile_width(int bn)
     g_force_bn = bn;
     return SSTE_OK;
 }
-#ifdef SSTE_PROBE
-extern "C" void sste_probe_set_mode(int mode) { g_probe_mode = mode; }
-extern "C" void sste_probe_set_dbg(long long *dbg) { g_probe_dbg = dbg; }
-#endif
 
 extern "C" sste_status sste_linear_fwd(sste_ctx *ctx, const void *X, int T, const void *vals, const void *meta, int O,
                                        int I, sste_dtype opdt, const float *out_scale_dev, void *Y, sste_dtype ydt,

@@ -31,6 +31,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_B
 
 constexpr int MAX_DEVICES = 64;
 void *g_scratch_addr[MAX_DEVICES] = {};   // device address of g_static_scratch, per device
+int g_device_major[MAX_DEVICES] = {};     // compute-capability major of the device, looked up with the address
 std::mutex g_setup_mutex;
 
 __device__ __forceinline__ double warp_sum_f64(double v)
@@ -109,10 +110,17 @@ beta_static_kernel(const uint4 *__restrict__ W, int I, unsigned char *__restrict
     }
 }
 
-// Device address of the scratch array on the current device.  Looked up once per device.
+// Device address of the scratch array on the current device.  Looked up once per device, together with
+// the device's architecture (the kernel image exists for compute capability 10.x only).
 sste_status scratch_address(int device, unsigned char **out)
 {
     std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!g_device_major[device]) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) return SSTE_ERR_CUDA;
+        g_device_major[device] = major;
+    }
+    if (g_device_major[device] != 10) return SSTE_ERR_ARCH;
     if (!g_scratch_addr[device]) {
         void *addr = nullptr;
         if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return SSTE_ERR_CUDA;
@@ -140,6 +148,12 @@ extern "C" sste_status sste_beta_init_static(int device, const void *W, int O, i
     if (st != SSTE_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     SSTE_CUDA_TRY(cudaMemsetAsync(scratch, 0, sizeof(unsigned int), s));   // the ticket counter starts at zero
-    beta_static_kernel<<<static_cast<unsigned int>(tiles), 256, 0, s>>>(static_cast<const uint4 *>(W), I, scratch, beta_dev);
-    return cudaGetLastError() == cudaSuccess ? SSTE_OK : SSTE_ERR_CUDA;
+    // the launch's own return code: an earlier, unrelated sticky error is not reported as this call's
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned int>(tiles));
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    SSTE_CUDA_TRY(cudaLaunchKernelEx(&cfg, beta_static_kernel, static_cast<const uint4 *>(W), I, scratch, beta_dev));
+    sste_count_launches(1);
+    return SSTE_OK;
 }

@@ -2,9 +2,10 @@
 library-chosen tile widths and split-K).
 
 Config 2 (GPT-2-small MLP): everything compared in full -- projection, metadata, MVUE bit for bit, the three
-products against complete fp64 products.  Config 3 (one GPT-2-large layer) and config 5 (one 7B-shaped FFN
-layer, FP8): the elementwise outputs in full, the products on a seeded sample of 256 output rows each, computed
-one by one as fp64 dot products of the decoded operands.
+products against complete fp64 products.  Every layer of config 3 (GPT-2-large block linears), the attention
+linears of config 4 and every layer of config 5 (7B-shaped FFN, FP8): the elementwise outputs in full, the
+products on a seeded sample of 256 output rows each, computed one by one as fp64 dot products of the decoded
+operands.
 """
 import numpy as np
 import pytest
@@ -85,14 +86,17 @@ def _sampled_products(lin, X_dec, dY_dec, w_dec, vals, meta, gvals, gmeta, wdt, 
                           w_dec[os_])
 
 
-def test_config3_ffn_layer_sampled(ctx):
+def _bf16_layer_sampled(ctx, cfg_id, layer, rng_seed):
+    """One bf16 layer at full size: beta, projection, metadata and MVUE in full and bit for bit; the three
+    products on N_SAMPLE rows each against fp64 dot products."""
     from paper_2409_09099_b200 import binding as B
-    cfg = synth.CONFIGS[3]
-    layer = 2                                           # fc1: W[5120, 1280], 16384 tokens
-    W, X, dY = synth.layer_tensors(3, layer)
+    cfg = synth.CONFIGS[cfg_id]
+    W, X, dY = synth.layer_tensors(cfg_id, layer)
     O, I = W.shape
     T = X.shape[0]
     lin = _run_layer(ctx, W, X, dY, layer, cfg["seed"], 0, False)
+    beta_ref = orc.beta(W)[0]
+    assert abs(lin.beta.item() - beta_ref) <= 1e-6 * beta_ref
     ov, om, od = orc.project_compress(W, np.float32(lin.beta.item()))
     assert np.array_equal(bits16(lin.vals), ov) and np.array_equal(bits16(lin.w_dense), od)
     assert np.array_equal(canonical_meta(ctx, lin.meta, O, I, B.BF16), om)
@@ -100,13 +104,28 @@ def test_config3_ffn_layer_sampled(ctx):
     assert np.array_equal(bits16(lin.gvals), ogv)
     assert np.array_equal(canonical_meta(ctx, lin.gmeta, O, T, B.BF16), ogm)
     _sampled_products(lin, orc.decode(X, orc.BF16), orc.decode(dY, orc.BF16), orc.decode(od, orc.BF16), ov, om, ogv, ogm,
-                      orc.BF16, orc.BF16, dict(xw=1.0, gw=1.0, gx=1.0), BF16_GEMM_TOL, np.random.default_rng(33))
+                      orc.BF16, orc.BF16, dict(xw=1.0, gw=1.0, gx=1.0), BF16_GEMM_TOL, np.random.default_rng(rng_seed))
 
 
-def test_config5_fp8_up_projection_sampled(ctx):
+# GPT-2-large block linears, 16384 tokens: qkv [3840, 1280], proj [1280, 1280], fc1 [5120, 1280], fc2 [1280, 5120]
+@pytest.mark.parametrize("layer", [0, 1, 2, 3])
+def test_config3_every_layer_sampled(ctx, layer):
+    _bf16_layer_sampled(ctx, 3, layer, 30 + layer)
+
+
+# the attention linears of a GPT-2-124M block, 8192 tokens: qkv [2304, 768], proj [768, 768] (its MLP layers have
+# the shapes of config 2, which is compared in full above)
+@pytest.mark.parametrize("layer", [0, 1])
+def test_config4_attention_linears_sampled(ctx, layer):
+    _bf16_layer_sampled(ctx, 4, layer, 40 + layer)
+
+
+# FP8 whole-process, 7B-shaped FFN, 16384 tokens: up / gate [11008, 4096] and down [4096, 11008] (K = 11008: an odd
+# number of pipeline stages and its own tile-width / split plan)
+@pytest.mark.parametrize("layer", [0, 1, 2])
+def test_config5_fp8_every_layer_sampled(ctx, layer):
     from paper_2409_09099_b200 import binding as B
     cfg = synth.CONFIGS[5]
-    layer = 0                                           # W_up[11008, 4096], 16384 tokens, FP8 whole-process
     W, X, dY = synth.layer_tensors(5, layer)
     O, I = W.shape
     T = X.shape[0]
@@ -127,4 +146,4 @@ def test_config5_fp8_up_projection_sampled(ctx):
     assert np.array_equal(canonical_meta(ctx, lin.gmeta, O, T, B.E5M2), ogm)
     inv = dict(xw=1.0 / (float(sx) * float(sw)), gw=1.0 / (float(sg) * float(sw)), gx=1.0 / (float(sg) * float(sx)))
     _sampled_products(lin, orc.decode(Xq, orc.E4M3), orc.decode(odq, orc.E5M2), orc.decode(od, orc.E4M3), ov, om, ogv, ogm,
-                      orc.E4M3, orc.E5M2, inv, FP8_GEMM_TOL, np.random.default_rng(55))
+                      orc.E4M3, orc.E5M2, inv, FP8_GEMM_TOL, np.random.default_rng(50 + layer))
