@@ -10,7 +10,7 @@
  *                 sste_mvue_sparsify      MVUE(grad_Z^T)        2:4 along tokens      (Sec. 5.1)
  *                 sste_linear_bwd_weight  grad_W = MVUE(grad_Z^T) X   sparse          (Sec. 5.1)
  *                 sste_linear_bwd_input   grad_X = grad_Z w~          dense           (Sec. 5.1)
- *   FP8 variant   sste_amax, sste_fp8_scale, sste_quantize_fp8 + the E4M3/E5M2 dtypes (Sec. 5.2)
+ *   FP8 variant   sste_amax, sste_project_amax, sste_quantize_fp8 + the E4M3/E5M2 dtypes (Sec. 5.2)
  *
  * Conventions (all entry points)
  *   - Every tensor pointer is DEVICE memory owned by the caller, row-major and
@@ -37,6 +37,12 @@
  *     with that product's output incomplete: poll before trusting results.
  *   - bf16 tensors hold IEEE bfloat16 bit patterns, E4M3 is the "fn" flavour
  *     (max 448, no infinity), E5M2 is IEEE-like (max finite 57344).
+ *   - FP8 per-tensor scaling (Sec. 5.2, "per-tensor rescaling before casting"): a tensor x is quantised as
+ *     q = cast(fl32(x * s)), s = fl32(fp8_max / amax(x)) (s = 1 if amax(x) = 0).  The state of a quantised tensor
+ *     is its AMAX, one device float: every call that quantises, or that consumes a quantised operand, takes the
+ *     `*_amax_dev` pointer and forms s itself with exactly these operations (so no separate kernel computes scales
+ *     or their products); a product multiplies its fp32 accumulator by fl32(fl32(1/s_a) * fl32(1/s_b)).  With bf16
+ *     operands these pointers are NULL.
  *
  * Compressed 2:4 operand ("vals" + "meta") of a logical [rows, K] matrix whose
  * groups of four run along K:
@@ -117,25 +123,29 @@ sste_status sste_beta_init(sste_ctx *ctx, const void *W, int O, int I, sste_dtyp
 /*
  * Eq. 4 + Sec. 4.2: w~ = beta * S_soft(w).  Per group of four along I, t = 2nd-smallest |w|,
  * s = sign(w) * max(|w| - t, 0) (one fp32 subtraction), w~ = fl32(s * beta)
- * [FP8: fl32(w~ * wscale)], one round-to-nearest-even cast to `odt` (E4M3: saturating).
+ * [FP8: fl32(w~ * s_w)], one round-to-nearest-even cast to `odt` (E4M3: saturating).
  * Pruned entries are +0.  Kept positions: rank by (|w| descending, index ascending), keep two.
- * W: bf16 [O, I].  odt: SSTE_BF16 or SSTE_E4M3.  wscale_dev: device float, NULL for bf16.
- * Outputs: vals [O, I/2] and meta (see top); dense_out (nullable) [O, I] in odt, the operand
- * of sste_linear_bwd_input.
+ * W: bf16 [O, I].  odt: SSTE_BF16 or SSTE_E4M3.  w_amax_dev: device float holding max|w~| of the bf16
+ * projection (from sste_project_amax), from which s_w is formed; NULL for bf16.
+ * Outputs: vals [O, I/2] and meta (see top); dense_out (nullable) [O, I] in odt: the dense copy of w~.
+ * sste_linear_bwd_input can work from (vals, meta) alone, so the dense copy is optional.
  */
 sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
-                                  const float *beta_dev, const float *wscale_dev, sste_dtype odt,
+                                  const float *beta_dev, const float *w_amax_dev, sste_dtype odt,
                                   void *vals, void *meta, void *dense_out, void *stream);
 
 /*
  * Sec. 5.1: Z = X S(W)^T on sparse tensor cores.  X [T, I], (vals, meta) the compressed w~
  * [O, I], both of dtype opdt (SSTE_BF16, or SSTE_E4M3 for the FP8 variant).  fp32 accumulation.
- * Y [T, O] of dtype ydt (SSTE_BF16 or SSTE_F32) = acc * out_scale, out_scale = *out_scale_dev
- * (NULL means 1; the FP8 variant passes 1/(sx*sw)).
+ * Y [T, O] of dtype ydt (SSTE_BF16 or SSTE_F32) = acc [* 1/s_x * 1/s_w for E4M3 operands: x_amax_dev and
+ * w_amax_dev are then the amax X and w~ were quantised with; both NULL for bf16, else SSTE_ERR_INVALID_ARG].
+ * y_amax_out_dev (nullable, device float): receives max|Y| of the stored output (the call zeroes it on the
+ * stream, the epilogue raises it by atomic maximum), so that a following layer that quantises Y needs no
+ * separate amax pass.
  */
 sste_status sste_linear_fwd(sste_ctx *ctx, const void *X, int T, const void *vals, const void *meta,
-                            int O, int I, sste_dtype opdt, const float *out_scale_dev,
-                            void *Y, sste_dtype ydt, void *stream);
+                            int O, int I, sste_dtype opdt, const float *x_amax_dev, const float *w_amax_dev,
+                            void *Y, sste_dtype ydt, float *y_amax_out_dev, void *stream);
 
 /*
  * Sec. 5.1: minimum-variance unbiased 2:4 sparsification of grad_Z^T (the paper applies MVUE to
@@ -147,34 +157,44 @@ sste_status sste_linear_fwd(sste_ctx *ctx, const void *X, int T, const void *val
  * shard, a multiple of 4, so that the draws do not depend on how the batch is sharded).
  * Philox4x32-10 with counter (lo32(g>>2), hi32(g>>2), tensor_id, step) and key
  * (lo32(seed), hi32(seed)); the group uses output word g&3, u = (word >> 8) * 2^-24.
- * dY: bf16 [T, O].  odt: SSTE_BF16, or SSTE_E5M2 with values fl32(v * gscale) (gscale_dev
- * non-NULL).  Outputs: the compressed operand of the TRANSPOSED matrix, logical [O, T]:
- * gvals [O, T/2], gmeta (see top).  dense_q_out (nullable, FP8 only): E5M2(fl32(dY * gscale)) [T, O].
+ * dY: bf16 [T, O].  odt: SSTE_BF16, or SSTE_E5M2 with values fl32(v * s_g), s_g formed from
+ * *g_amax_dev = max|dY| (non-NULL then).  Outputs: the compressed operand of the TRANSPOSED matrix, logical
+ * [O, T]: gvals [O, T/2], gmeta (see top).  dense_q_out (nullable, FP8 only): E5M2(fl32(dY * s_g)) [T, O].
+ * counter_cols: the number of columns the group index counts with, g = (token_offset/4 + tg)*counter_cols + j;
+ * 0 means O.  A caller that padded O up to a multiple of 128 passes the unpadded column count, so that the draws
+ * of the real columns are those of the unpadded problem (columns j >= counter_cols must be all zero: a zero
+ * group yields zeros whatever its draw).
  */
 sste_status sste_mvue_sparsify(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt,
                                uint64_t seed, uint32_t tensor_id, uint32_t step, uint64_t token_offset,
-                               const float *gscale_dev, sste_dtype odt,
+                               int counter_cols, const float *g_amax_dev, sste_dtype odt,
                                void *gvals, void *gmeta, void *dense_q_out, void *stream);
 
 /*
  * Sec. 5.1: grad_X = grad_Z S(W), a dense product (the 2:4 structure of S(W) lies along I, which
- * is not the reduction dimension here).  dY [T, O] of dtype gdt (SSTE_BF16 / SSTE_E5M2),
- * Wt_dense [O, I] of dtype wdt (SSTE_BF16 / SSTE_E4M3) as written by sste_project_compress.
- * dX [T, I] of dtype xdt = acc * out_scale.
+ * is not the reduction dimension here).  dY [T, O] of dtype gdt (SSTE_BF16 / SSTE_E5M2).  S(W) [O, I] of
+ * dtype wdt (SSTE_BF16 / SSTE_E4M3) is given EITHER as the dense copy Wt_dense written by
+ * sste_project_compress, OR (Wt_dense = NULL) as the forward's compressed operand (vals, meta): the kernel then
+ * expands each K slice into the dense shared-memory operand itself (+0 in the pruned positions), the same
+ * product bit for bit, and the dense copy need not exist.  dX [T, I] of dtype xdt = acc [* 1/s_g * 1/s_w for FP8
+ * operands, from g_amax_dev / w_amax_dev; NULL for bf16].  dx_amax_out_dev: nullable, max|dX| as for the forward.
  */
 sste_status sste_linear_bwd_input(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt,
-                                  const void *Wt_dense, int I, sste_dtype wdt,
-                                  const float *out_scale_dev, void *dX, sste_dtype xdt, void *stream);
+                                  const void *Wt_dense, const void *vals, const void *meta, int I, sste_dtype wdt,
+                                  const float *g_amax_dev, const float *w_amax_dev,
+                                  void *dX, sste_dtype xdt, float *dx_amax_out_dev, void *stream);
 
 /*
  * Sec. 5.1: grad_W = MVUE(grad_Z^T) X on sparse tensor cores.  (gvals, gmeta) logical [O, T] of
  * dtype gdt (SSTE_BF16 / SSTE_E5M2) from sste_mvue_sparsify, X [T, I] of dtype xdt
- * (SSTE_BF16 / SSTE_E4M3).  dW [O, I] of dtype dwdt (SSTE_BF16 or SSTE_F32) = acc * out_scale.
+ * (SSTE_BF16 / SSTE_E4M3).  dW [O, I] of dtype dwdt (SSTE_BF16 or SSTE_F32) = acc [* 1/s_g * 1/s_x for FP8
+ * operands, from g_amax_dev / x_amax_dev; NULL for bf16].
  * Straight-through estimator (Eq. 3): this gradient is applied to the dense weight unchanged.
  */
 sste_status sste_linear_bwd_weight(sste_ctx *ctx, const void *gvals, const void *gmeta, int O, int T,
                                    sste_dtype gdt, const void *X, int I, sste_dtype xdt,
-                                   const float *out_scale_dev, void *dW, sste_dtype dwdt, void *stream);
+                                   const float *g_amax_dev, const float *x_amax_dev,
+                                   void *dW, sste_dtype dwdt, void *stream);
 
 /*
  * The same beta as sste_beta_init, for callers that cannot allocate device memory at all (the paper has
@@ -212,16 +232,15 @@ sste_status sste_amax(sste_ctx *ctx, const void *x, size_t n, sste_dtype dt, flo
 sste_status sste_project_amax(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, const float *beta_dev,
                               float *amax_dev, void *stream);
 
-/* *scale_dev = fl32(fp8_max(odt) / *amax_dev) (1 if amax is 0); *inv_scale_dev (nullable) = fl32(1 / scale). */
+/* Inspection helper (no call of the path needs it: they form the scale from the amax themselves):
+ * *scale_dev = fl32(fp8_max(odt) / *amax_dev) (1 if amax is 0); *inv_scale_dev (nullable) = fl32(1 / scale). */
 sste_status sste_fp8_scale(sste_ctx *ctx, const float *amax_dev, sste_dtype odt, float *scale_dev,
                            float *inv_scale_dev, void *stream);
 
-/* q = cast_rn_satfinite(fl32(x * scale)), x bf16, q E4M3 or E5M2; n % 16 == 0. */
-sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n, const float *scale_dev,
+/* q = cast_rn_satfinite(fl32(x * s)), s formed from *amax_dev = max|x| (see top); x bf16, q E4M3 or E5M2;
+ * n % 16 == 0. */
+sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n, const float *amax_dev,
                               sste_dtype odt, void *q, void *stream);
-
-/* *out_dev = fl32(fl32(a * b)) for two device scalars (e.g. the product of two inverse scales). */
-sste_status sste_scalar_mul(sste_ctx *ctx, const float *a_dev, const float *b_dev, float *out_dev, void *stream);
 
 /* ---- ablation variants of the pruning step (the axes of the paper's ablations; not on the default path) ---- */
 
@@ -237,7 +256,7 @@ typedef enum { SSTE_PRUNE_SOFT = 0, SSTE_PRUNE_HARD = 1 } sste_pruning;
  * errors as sste_project_compress; SSTE_ERR_INVALID_ARG for an unknown pruning or gamma outside [0, 1].
  */
 sste_status sste_project_compress_variant(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
-                                          const float *beta_dev, const float *wscale_dev, sste_dtype odt,
+                                          const float *beta_dev, const float *w_amax_dev, sste_dtype odt,
                                           sste_pruning pruning, float gamma, void *vals, void *meta,
                                           void *dense_out, void *stream);
 
@@ -268,7 +287,30 @@ sste_status sste_srste_decay(sste_ctx *ctx, const void *W, const void *meta, int
 sste_status sste_flip_count(sste_ctx *ctx, const void *meta_prev, const void *meta_cur, int rows, int k,
                             unsigned long long *count_dev, void *stream);
 
+/* ---- shapes that are not multiples of 128 ---- */
+
+/*
+ * Every call above wants O, I and T to be multiples of 128.  Other shapes (a 50257-row vocabulary projection,
+ * a batch of 1000 tokens) are run on zero-padded copies: a group of four zeros is a fixed point of Eq. 4 and of
+ * the MVUE rule, contributes nothing to beta (Eq. 5), to an amax or to a product, so the results on the real
+ * rows and columns are those of the unpadded problem (for MVUE pass counter_cols = the unpadded column count).
+ * sste_padded_dim(n) = the next multiple of 128.  sste_pad_2d copies src [rows, cols] into the top-left corner
+ * of dst [rows_p, cols_p] (rows_p >= rows, cols_p >= cols, cols_p % 8 == 0, dst 16-byte aligned) and zero-fills
+ * the rest; sste_crop_2d copies the top-left [rows, cols] corner of src [rows_p, cols_p] into dst [rows, cols].
+ * Elements are 2 bytes (bf16).  Both are single passes over the larger tensor.
+ */
+int sste_padded_dim(int n);
+sste_status sste_pad_2d(sste_ctx *ctx, const void *src, int rows, int cols, void *dst, int rows_p, int cols_p,
+                        void *stream);
+sste_status sste_crop_2d(sste_ctx *ctx, const void *src, int rows_p, int cols_p, void *dst, int rows, int cols,
+                         void *stream);
+
 /* ---- test / debug helpers ---- */
+
+/* Compressed operand (vals [rows, k/2] + metadata image) -> dense [rows, k] of the same dtype dt (SSTE_BF16,
+ * SSTE_E4M3 or SSTE_E5M2), +0 in the pruned positions: the matrix the sparse tensor-core instruction sees. */
+sste_status sste_decompress(sste_ctx *ctx, const void *vals, const void *meta, int rows, int k, sste_dtype dt,
+                            void *dense_out, void *stream);
 
 /* Operand-image metadata -> canonical uint16 [rows, k/16] (see top).  dt selects the 16-bit or 8-bit image. */
 sste_status sste_meta_to_canonical(sste_ctx *ctx, const void *meta, int rows, int k, sste_dtype dt,
@@ -282,7 +324,7 @@ unsigned long long sste_debug_launch_count(void);
 /* The three products pick the width of their output tiles (128, 192 or 256 columns) from the problem
  * shape.  This process-wide hook pins it so that tests can cover every variant; widths a product does
  * not support (192 needs a K-major B operand, i.e. the forward) fall back to the automatic choice.
- * bn: 0 (automatic), 128, 192 or 256; anything else gives SSTE_ERR_INVALID_ARG. */
+ * bn: 0 (automatic), 128, 192, 224 (forward only) or 256; anything else gives SSTE_ERR_INVALID_ARG. */
 sste_status sste_debug_force_tile_width(int bn);
 /* Same for the split-K factor: 0 (automatic) or 1..4; a factor the shape or the workspace does not allow
  * falls back to the automatic choice. */

@@ -27,9 +27,10 @@ EXPORTS = [
     "sste_workspace_bytes", "sste_create", "sste_destroy", "sste_status_string", "sste_poll_device_status",
     "sste_vals_bytes", "sste_meta_bytes", "sste_beta_init", "sste_project_compress", "sste_linear_fwd",
     "sste_mvue_sparsify", "sste_linear_bwd_input", "sste_linear_bwd_weight", "sste_amax", "sste_fp8_scale",
-    "sste_quantize_fp8", "sste_scalar_mul", "sste_meta_to_canonical", "sste_debug_force_tile_width", "sste_debug_force_splits",
+    "sste_quantize_fp8", "sste_meta_to_canonical", "sste_debug_force_tile_width", "sste_debug_force_splits",
     "sste_workspace_bytes_recommended", "sste_beta_init_static", "sste_debug_launch_count", "sste_flip_count",
     "sste_project_compress_variant", "sste_beta_init_l1", "sste_srste_decay", "sste_project_amax",
+    "sste_decompress", "sste_padded_dim", "sste_pad_2d", "sste_crop_2d",
 ]
 
 
@@ -67,6 +68,11 @@ def _ptr(t):
 
 def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def padded_dim(n: int) -> int:
+    """sste_padded_dim: the next multiple of 128."""
+    return int(load().sste_padded_dim(n))
 
 
 def launch_count() -> int:
@@ -124,41 +130,45 @@ class Context:
         O, I = W.shape
         self._check(self.lib.sste_beta_init(self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev), _stream()))
 
-    def project_compress(self, W, beta_dev, vals, meta, dense_out=None, wscale_dev=None):
+    def project_compress(self, W, beta_dev, vals, meta, dense_out=None, w_amax_dev=None):
         O, I = W.shape
         self._check(self.lib.sste_project_compress(
-            self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev), _ptr(wscale_dev), _CODE_OF[vals.dtype],
+            self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev), _ptr(w_amax_dev), _CODE_OF[vals.dtype],
             _ptr(vals), _ptr(meta), _ptr(dense_out), _stream()))
 
-    def linear_fwd(self, X, vals, meta, Y, out_scale_dev=None):
+    def linear_fwd(self, X, vals, meta, Y, x_amax_dev=None, w_amax_dev=None, y_amax_out_dev=None):
         T, I = X.shape
         O = vals.shape[0]
         self._check(self.lib.sste_linear_fwd(
-            self.handle, _ptr(X), T, _ptr(vals), _ptr(meta), O, I, _CODE_OF[X.dtype], _ptr(out_scale_dev),
-            _ptr(Y), _CODE_OF[Y.dtype], _stream()))
+            self.handle, _ptr(X), T, _ptr(vals), _ptr(meta), O, I, _CODE_OF[X.dtype], _ptr(x_amax_dev),
+            _ptr(w_amax_dev), _ptr(Y), _CODE_OF[Y.dtype], _ptr(y_amax_out_dev), _stream()))
 
-    def mvue_sparsify(self, dY, seed, tensor_id, step, gvals, gmeta, dense_q_out=None, gscale_dev=None,
-                      token_offset=0):
+    def mvue_sparsify(self, dY, seed, tensor_id, step, gvals, gmeta, dense_q_out=None, g_amax_dev=None,
+                      token_offset=0, counter_cols=0):
         T, O = dY.shape
         self._check(self.lib.sste_mvue_sparsify(
             self.handle, _ptr(dY), T, O, _CODE_OF[dY.dtype], ctypes.c_uint64(seed), ctypes.c_uint32(tensor_id),
-            ctypes.c_uint32(step), ctypes.c_uint64(token_offset), _ptr(gscale_dev), _CODE_OF[gvals.dtype],
-            _ptr(gvals), _ptr(gmeta),
-            _ptr(dense_q_out), _stream()))
+            ctypes.c_uint32(step), ctypes.c_uint64(token_offset), ctypes.c_int(counter_cols), _ptr(g_amax_dev),
+            _CODE_OF[gvals.dtype], _ptr(gvals), _ptr(gmeta), _ptr(dense_q_out), _stream()))
 
-    def linear_bwd_input(self, dY, Wt_dense, dX, out_scale_dev=None):
+    def linear_bwd_input(self, dY, Wt_dense, dX, g_amax_dev=None, w_amax_dev=None, vals=None, meta=None,
+                         dx_amax_out_dev=None):
+        """grad_X from the dense copy `Wt_dense`, or (Wt_dense=None) from the compressed operand (vals, meta)."""
         T, O = dY.shape
-        I = Wt_dense.shape[1]
+        if Wt_dense is not None:
+            I, wdt = Wt_dense.shape[1], _CODE_OF[Wt_dense.dtype]
+        else:
+            I, wdt = 2 * vals.shape[1], _CODE_OF[vals.dtype]
         self._check(self.lib.sste_linear_bwd_input(
-            self.handle, _ptr(dY), T, O, _CODE_OF[dY.dtype], _ptr(Wt_dense), I, _CODE_OF[Wt_dense.dtype],
-            _ptr(out_scale_dev), _ptr(dX), _CODE_OF[dX.dtype], _stream()))
+            self.handle, _ptr(dY), T, O, _CODE_OF[dY.dtype], _ptr(Wt_dense), _ptr(vals), _ptr(meta), I, wdt,
+            _ptr(g_amax_dev), _ptr(w_amax_dev), _ptr(dX), _CODE_OF[dX.dtype], _ptr(dx_amax_out_dev), _stream()))
 
-    def linear_bwd_weight(self, gvals, gmeta, X, dW, out_scale_dev=None):
+    def linear_bwd_weight(self, gvals, gmeta, X, dW, g_amax_dev=None, x_amax_dev=None):
         O = gvals.shape[0]
         T, I = X.shape
         self._check(self.lib.sste_linear_bwd_weight(
             self.handle, _ptr(gvals), _ptr(gmeta), O, T, _CODE_OF[gvals.dtype], _ptr(X), I, _CODE_OF[X.dtype],
-            _ptr(out_scale_dev), _ptr(dW), _CODE_OF[dW.dtype], _stream()))
+            _ptr(g_amax_dev), _ptr(x_amax_dev), _ptr(dW), _CODE_OF[dW.dtype], _stream()))
 
     # ---- FP8 helpers ----------------------------------------------------------------------------
 
@@ -175,20 +185,17 @@ class Context:
         self._check(self.lib.sste_fp8_scale(self.handle, _ptr(amax_dev), odt, _ptr(scale_dev), _ptr(inv_scale_dev),
                                             _stream()))
 
-    def quantize_fp8(self, x, scale_dev, q):
-        self._check(self.lib.sste_quantize_fp8(self.handle, _ptr(x), ctypes.c_size_t(x.numel()), _ptr(scale_dev),
+    def quantize_fp8(self, x, amax_dev, q):
+        self._check(self.lib.sste_quantize_fp8(self.handle, _ptr(x), ctypes.c_size_t(x.numel()), _ptr(amax_dev),
                                                _CODE_OF[q.dtype], _ptr(q), _stream()))
-
-    def scalar_mul(self, a_dev, b_dev, out_dev):
-        self._check(self.lib.sste_scalar_mul(self.handle, _ptr(a_dev), _ptr(b_dev), _ptr(out_dev), _stream()))
 
     # ---- ablation variants of the pruning step ---------------------------------------------------
 
-    def project_compress_variant(self, W, beta_dev, vals, meta, dense_out=None, wscale_dev=None, hard=False,
+    def project_compress_variant(self, W, beta_dev, vals, meta, dense_out=None, w_amax_dev=None, hard=False,
                                  gamma=0.0):
         O, I = W.shape
         self._check(self.lib.sste_project_compress_variant(
-            self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev), _ptr(wscale_dev), _CODE_OF[vals.dtype],
+            self.handle, _ptr(W), O, I, _CODE_OF[W.dtype], _ptr(beta_dev), _ptr(w_amax_dev), _CODE_OF[vals.dtype],
             PRUNE_HARD if hard else PRUNE_SOFT, ctypes.c_float(gamma), _ptr(vals), _ptr(meta), _ptr(dense_out),
             _stream()))
 
@@ -210,6 +217,21 @@ class Context:
                                              _stream()))
 
     # ---- helpers --------------------------------------------------------------------------------
+
+    def decompress(self, vals, meta, dense_out):
+        rows, k = dense_out.shape
+        self._check(self.lib.sste_decompress(self.handle, _ptr(vals), _ptr(meta), rows, k, _CODE_OF[vals.dtype],
+                                             _ptr(dense_out), _stream()))
+
+    def pad_2d(self, src, dst):
+        """dst[:rows, :cols] = src, zeros elsewhere (2-byte elements)."""
+        self._check(self.lib.sste_pad_2d(self.handle, _ptr(src), src.shape[0], src.shape[1], _ptr(dst), dst.shape[0],
+                                         dst.shape[1], _stream()))
+
+    def crop_2d(self, src, dst):
+        """dst = src[:rows, :cols] (2-byte elements)."""
+        self._check(self.lib.sste_crop_2d(self.handle, _ptr(src), src.shape[0], src.shape[1], _ptr(dst), dst.shape[0],
+                                          dst.shape[1], _stream()))
 
     def meta_to_canonical(self, meta, rows, k, dt, out):
         self._check(self.lib.sste_meta_to_canonical(self.handle, _ptr(meta), rows, k, dt, _ptr(out), _stream()))

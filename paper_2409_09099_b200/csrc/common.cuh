@@ -75,6 +75,22 @@ __device__ __forceinline__ uint32_t sste_f32_to_e5m2(float f)
     return static_cast<uint32_t>(__nv_cvt_float_to_fp8(f, __NV_SATFINITE, __NV_E5M2));
 }
 
+// FP8 per-tensor scaling (Sec. 5.2): scale = fp8_max / amax, 1 for an all-zero tensor.  Every kernel that
+// quantises or rescales forms the scale from the tensor's amax with exactly these single-rounded operations.
+__device__ __forceinline__ float sste_scale_from_amax(float amax, float fp8_max)
+{
+    return (amax == 0.0f) ? 1.0f : __fdiv_rn(fp8_max, amax);
+}
+// factor that undoes the scales of two quantised operands in a product's epilogue: fl(fl(1/sa) * fl(1/sb))
+__device__ __forceinline__ float sste_out_scale(const float *a_amax, float a_fp8_max, const float *b_amax, float b_fp8_max)
+{
+    if (!a_amax || !b_amax) return 1.0f;
+    const float ia = __fdiv_rn(1.0f, sste_scale_from_amax(*a_amax, a_fp8_max));
+    const float ib = __fdiv_rn(1.0f, sste_scale_from_amax(*b_amax, b_fp8_max));
+    return __fmul_rn(ia, ib);
+}
+static inline float sste_fp8_max(sste_dtype dt) { return dt == SSTE_E4M3 ? 448.0f : dt == SSTE_E5M2 ? 57344.0f : 0.0f; }
+
 // Byte offset of (row m, K-offset k) inside a 2 KB metadata atom of 128 rows x 128 logical K.
 __device__ __host__ __forceinline__ uint32_t sste_meta_atom_byte16(uint32_t m, uint32_t k)
 {

@@ -81,7 +81,7 @@ __device__ __forceinline__ SoftGroup soft_group(uint32_t w01, uint32_t w23, floa
 template <bool FP8, int MODE>
 __global__ void __launch_bounds__(EW_THREADS)
 project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restrict__ beta_dev,
-                        const float *__restrict__ wscale_dev, float gamma, void *__restrict__ vals,
+                        const float *__restrict__ w_amax_dev, float gamma, void *__restrict__ vals,
                         uint8_t *__restrict__ meta, void *__restrict__ dense)
 {
     __shared__ __align__(16) uint8_t meta_s[512];
@@ -90,7 +90,7 @@ project_compress_kernel(const uint4 *__restrict__ W, int I, const float *__restr
     sste_pdl_trigger();
     sste_pdl_wait();
     const float beta = *beta_dev;
-    const float wscale = FP8 ? *wscale_dev : 1.0f;
+    const float wscale = FP8 ? sste_scale_from_amax(*w_amax_dev, 448.0f) : 1.0f;
     const size_t row_chunks = static_cast<size_t>(I) / 8;
 
     uint4 in[PC_CHUNKS];
@@ -336,10 +336,13 @@ __device__ __forceinline__ MvueGroup mvue_group(uint32_t p01, uint32_t p23, floa
 // One CTA: 128 tokens x 128 output columns of dY.  A thread task is 4 tokens x 8 columns
 // (8 groups, two Philox calls); results are transposed through shared memory so that every
 // output row (= column of dY) receives whole 128-byte lines.
-template <bool FP8>
+// ANY_COUNTER: counter_cols is not a multiple of 4 (a padded, odd column count), so a thread's eight
+// consecutive group indices do not start on a Philox block and span three blocks instead of two.
+template <bool FP8, bool ANY_COUNTER>
 __global__ void __launch_bounds__(EW_THREADS, 4)
 mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t key1, uint32_t tensor_id,
-            uint32_t step, uint64_t tg_offset, const float *__restrict__ gscale_dev, void *__restrict__ gvals,
+            uint32_t step, uint64_t tg_offset, uint32_t counter_cols, const float *__restrict__ g_amax_dev,
+            void *__restrict__ gvals,
             uint8_t *__restrict__ gmeta, void *__restrict__ dense_q)
 {
     // bf16: 128 rows x 32 words; fp8: 128 rows x 16 words
@@ -349,7 +352,7 @@ mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t 
     const int jb = blockIdx.x, tb = blockIdx.y;   // column block, token block
     sste_pdl_trigger();
     sste_pdl_wait();
-    const float gscale = FP8 ? *gscale_dev : 1.0f;
+    const float gscale = FP8 ? sste_scale_from_amax(*g_amax_dev, 57344.0f) : 1.0f;
     const size_t row_chunks = static_cast<size_t>(O) / 8;
 
 #pragma unroll
@@ -362,13 +365,25 @@ mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t 
 #pragma unroll
         for (int i = 0; i < 4; ++i) in[i] = __ldg(dY + (tok0 + i) * row_chunks + jb * 16 + jc);
 
-        const uint64_t g0 = (tg_offset + static_cast<uint64_t>(tb) * 32 + tgl) * static_cast<uint64_t>(O) +
+        const uint64_t g0 = (tg_offset + static_cast<uint64_t>(tb) * 32 + tgl) * static_cast<uint64_t>(counter_cols) +
                             static_cast<uint64_t>(jb) * 128 + jc * 8;
         const uint64_t q = g0 >> 2;
         uint32_t rnd[8];
-        philox4x32_10(static_cast<uint32_t>(q), static_cast<uint32_t>(q >> 32), tensor_id, step, key0, key1, rnd);
-        philox4x32_10(static_cast<uint32_t>(q + 1), static_cast<uint32_t>((q + 1) >> 32), tensor_id, step, key0,
-                      key1, rnd + 4);
+        if (!ANY_COUNTER) {
+            philox4x32_10(static_cast<uint32_t>(q), static_cast<uint32_t>(q >> 32), tensor_id, step, key0, key1, rnd);
+            philox4x32_10(static_cast<uint32_t>(q + 1), static_cast<uint32_t>((q + 1) >> 32), tensor_id, step, key0,
+                          key1, rnd + 4);
+        } else {
+            uint32_t r12[12];
+#pragma unroll
+            for (int b = 0; b < 3; ++b)
+                philox4x32_10(static_cast<uint32_t>(q + b), static_cast<uint32_t>((q + b) >> 32), tensor_id, step, key0,
+                              key1, r12 + 4 * b);
+            const uint32_t sh = static_cast<uint32_t>(g0) & 3u;     // group g0 + e uses word (g0 + e) & 3 of block (g0 + e) >> 2
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                rnd[e] = sh == 0 ? r12[e] : sh == 1 ? r12[e + 1] : sh == 2 ? r12[e + 2] : r12[e + 3];
+        }
 
         const uint32_t raw[4][4] = {{in[0].x, in[0].y, in[0].z, in[0].w},
                                     {in[1].x, in[1].y, in[1].z, in[1].w},
@@ -500,26 +515,19 @@ __global__ void fp8_scale_kernel(const float *amax_dev, float fp8_max, float *sc
     sste_pdl_trigger();
     sste_pdl_wait();
     const float a = *amax_dev;
-    const float s = (a == 0.0f) ? 1.0f : __fdiv_rn(fp8_max, a);
+    const float s = sste_scale_from_amax(a, fp8_max);
     *scale_dev = s;
     if (inv_scale_dev) *inv_scale_dev = __fdiv_rn(1.0f, s);
 }
 
-__global__ void scalar_mul_kernel(const float *a, const float *b, float *out)
-{
-    sste_pdl_trigger();
-    sste_pdl_wait();
-    *out = __fmul_rn(*a, *b);
-}
-
 template <bool E5M2>
 __global__ void __launch_bounds__(EW_THREADS)
-quantize_kernel(const uint4 *__restrict__ x, size_t n_chunks, const float *__restrict__ scale_dev,
+quantize_kernel(const uint4 *__restrict__ x, size_t n_chunks, const float *__restrict__ amax_dev,
                 uint2 *__restrict__ q)
 {
     sste_pdl_trigger();
     sste_pdl_wait();
-    const float scale = *scale_dev;
+    const float scale = sste_scale_from_amax(*amax_dev, E5M2 ? 57344.0f : 448.0f);
     for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
          c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
         const uint4 v = __ldg(x + c);
@@ -556,6 +564,85 @@ meta_to_canonical_kernel(const uint8_t *__restrict__ meta, int rows, int k, uint
         const uint32_t b0 = EIGHT_BIT ? sste_meta_atom_byte8(m, ko) : sste_meta_atom_byte16(m, ko);
         const uint32_t b1 = EIGHT_BIT ? sste_meta_atom_byte8(m, ko + 8) : sste_meta_atom_byte16(m, ko + 8);
         out[w] = static_cast<uint16_t>(base[b0] | (base[b1] << 8));
+    }
+}
+
+// ---------------------------------------------------------------- compressed operand -> dense (test / debug)
+
+// One thread per 16 bytes of values: bf16 4 groups (16 dense elements), fp8 8 groups (32 dense elements).
+template <bool EIGHT_BIT>
+__global__ void __launch_bounds__(EW_THREADS)
+decompress_kernel(const uint4 *__restrict__ vals, const uint8_t *__restrict__ meta, int k, size_t n_units,
+                  uint4 *__restrict__ dense)
+{
+    sste_pdl_trigger();
+    sste_pdl_wait();
+    const size_t units_per_row = static_cast<size_t>(k) / (EIGHT_BIT ? 32 : 16);
+    for (size_t un = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; un < n_units;
+         un += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const uint32_t row = static_cast<uint32_t>(un / units_per_row);
+        const uint32_t kk = static_cast<uint32_t>(un % units_per_row) * (EIGHT_BIT ? 32u : 16u);
+        const uint8_t *atom = meta + (static_cast<size_t>(row >> 7) * (k / 128) + (kk >> 7)) * 2048;
+        const uint4 v = __ldg(vals + un);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[8];
+        if (EIGHT_BIT) {
+            const uint32_t codes = *reinterpret_cast<const uint32_t *>(atom + sste_meta_atom_byte8(row & 127u, kk & 127u));
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                const uint32_t nib = (codes >> (4 * g)) & 0xfu, p0 = nib & 3u, p1 = nib >> 2;
+                const uint32_t pr = (g & 1) ? (w[g >> 1] >> 16) : (w[g >> 1] & 0xffffu);
+                o[g] = ((pr & 0xffu) << (8 * p0)) | ((pr >> 8) << (8 * p1));
+            }
+        } else {
+            const uint32_t codes = *reinterpret_cast<const uint16_t *>(atom + sste_meta_atom_byte16(row & 127u, kk & 127u));
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const uint32_t nib = (codes >> (4 * g)) & 0xfu, p0 = nib & 3u, p1 = nib >> 2;
+                const uint64_t d = (static_cast<uint64_t>(w[g] & 0xffffu) << (16 * p0)) |
+                                   (static_cast<uint64_t>(w[g] >> 16) << (16 * p1));
+                o[2 * g] = static_cast<uint32_t>(d);
+                o[2 * g + 1] = static_cast<uint32_t>(d >> 32);
+            }
+        }
+        dense[2 * un] = make_uint4(o[0], o[1], o[2], o[3]);
+        dense[2 * un + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
+// ---------------------------------------------------------------- zero padding to multiples of 128 and back
+
+// dst [rows_p, cols_p] <- src [rows, cols] in the top-left corner, zeros elsewhere; 2-byte elements, one
+// thread per 8 destination elements (16-byte stores; element-wise loads, src rows need no alignment).
+__global__ void __launch_bounds__(EW_THREADS)
+pad_2d_kernel(const uint16_t *__restrict__ src, int rows, int cols, uint4 *__restrict__ dst, int cols_p, size_t n_vec)
+{
+    sste_pdl_trigger();
+    sste_pdl_wait();
+    const size_t vec_per_row = static_cast<size_t>(cols_p) / 8;
+    for (size_t v = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; v < n_vec;
+         v += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const size_t r = v / vec_per_row;
+        const int c0 = static_cast<int>(v % vec_per_row) * 8;
+        uint32_t e[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            e[i] = (r < static_cast<size_t>(rows) && c0 + i < cols) ? __ldg(src + r * cols + c0 + i) : 0u;
+        dst[v] = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
+    }
+}
+
+// dst [rows, cols] <- top-left corner of src [rows_p, cols_p]; one thread per element pair would be wasteful for
+// odd cols, so one thread per destination element (coalesced 2-byte accesses).
+__global__ void __launch_bounds__(EW_THREADS)
+crop_2d_kernel(const uint16_t *__restrict__ src, int cols_p, uint16_t *__restrict__ dst, int cols, size_t n)
+{
+    sste_pdl_trigger();
+    sste_pdl_wait();
+    for (size_t i = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; i < n;
+         i += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const size_t r = i / cols, c = i % cols;
+        dst[i] = __ldg(src + r * cols_p + c);
     }
 }
 
@@ -676,12 +763,12 @@ sste_status beta_launch(sste_ctx *ctx, const void *W, int O, int I, sste_dtype w
 
 // mode: 0 = the method's projection, 1 = interpolated threshold, 2 = hard thresholding
 sste_status project_launch(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt, const float *beta_dev,
-                           const float *wscale_dev, sste_dtype odt, int mode, float gamma, void *vals, void *meta,
+                           const float *w_amax_dev, sste_dtype odt, int mode, float gamma, void *vals, void *meta,
                            void *dense_out, void *stream)
 {
     if (!ctx || !W || !beta_dev || !vals || !meta) return SSTE_ERR_INVALID_ARG;
     if (wdt != SSTE_BF16 || (odt != SSTE_BF16 && odt != SSTE_E4M3)) return SSTE_ERR_DTYPE;
-    if (odt == SSTE_E4M3 && !wscale_dev) return SSTE_ERR_INVALID_ARG;
+    if (odt == SSTE_E4M3 && !w_amax_dev) return SSTE_ERR_INVALID_ARG;
     if (!sste_mult128(O) || !sste_mult128(I)) return SSTE_ERR_SHAPE;
     if (!sste_aligned(W, 128) || !sste_aligned(vals, 128) || !sste_aligned(meta, 128) ||
         !sste_aligned(dense_out, 128))
@@ -695,7 +782,7 @@ sste_status project_launch(sste_ctx *ctx, const void *W, int O, int I, sste_dtyp
     const bool f8 = (odt == SSTE_E4M3);
 #define SSTE_PC_LAUNCH(F8, MODE)                                                                                   \
     sste_launch(project_compress_kernel<F8, MODE>, dim3(grid), dim3(EW_THREADS), 0, s, w, I, beta_dev,           \
-                F8 ? wscale_dev : nullptr, gamma, vals, m, dense_out)
+                F8 ? w_amax_dev : nullptr, gamma, vals, m, dense_out)
     if (mode == 0) { if (f8) SSTE_PC_LAUNCH(true, 0); else SSTE_PC_LAUNCH(false, 0); }
     else if (mode == 1) { if (f8) SSTE_PC_LAUNCH(true, 1); else SSTE_PC_LAUNCH(false, 1); }
     else { if (f8) SSTE_PC_LAUNCH(true, 2); else SSTE_PC_LAUNCH(false, 2); }
@@ -718,21 +805,21 @@ extern "C" sste_status sste_beta_init_l1(sste_ctx *ctx, const void *W, int O, in
 }
 
 extern "C" sste_status sste_project_compress(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
-                                             const float *beta_dev, const float *wscale_dev, sste_dtype odt,
+                                             const float *beta_dev, const float *w_amax_dev, sste_dtype odt,
                                              void *vals, void *meta, void *dense_out, void *stream)
 {
-    return project_launch(ctx, W, O, I, wdt, beta_dev, wscale_dev, odt, 0, 0.0f, vals, meta, dense_out, stream);
+    return project_launch(ctx, W, O, I, wdt, beta_dev, w_amax_dev, odt, 0, 0.0f, vals, meta, dense_out, stream);
 }
 
 extern "C" sste_status sste_project_compress_variant(sste_ctx *ctx, const void *W, int O, int I, sste_dtype wdt,
-                                                     const float *beta_dev, const float *wscale_dev, sste_dtype odt,
+                                                     const float *beta_dev, const float *w_amax_dev, sste_dtype odt,
                                                      sste_pruning pruning, float gamma, void *vals, void *meta,
                                                      void *dense_out, void *stream)
 {
     if (pruning != SSTE_PRUNE_SOFT && pruning != SSTE_PRUNE_HARD) return SSTE_ERR_INVALID_ARG;
     if (!(gamma >= 0.0f && gamma <= 1.0f)) return SSTE_ERR_INVALID_ARG;
     const int mode = (pruning == SSTE_PRUNE_HARD) ? 2 : (gamma == 0.0f ? 0 : 1);
-    return project_launch(ctx, W, O, I, wdt, beta_dev, wscale_dev, odt, mode, gamma, vals, meta, dense_out, stream);
+    return project_launch(ctx, W, O, I, wdt, beta_dev, w_amax_dev, odt, mode, gamma, vals, meta, dense_out, stream);
 }
 
 extern "C" sste_status sste_srste_decay(sste_ctx *ctx, const void *W, const void *meta, int O, int I,
@@ -758,13 +845,15 @@ extern "C" sste_status sste_srste_decay(sste_ctx *ctx, const void *W, const void
 }
 
 extern "C" sste_status sste_mvue_sparsify(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt, uint64_t seed,
-                                          uint32_t tensor_id, uint32_t step, uint64_t token_offset,
-                                          const float *gscale_dev, sste_dtype odt, void *gvals, void *gmeta,
+                                          uint32_t tensor_id, uint32_t step, uint64_t token_offset, int counter_cols,
+                                          const float *g_amax_dev, sste_dtype odt, void *gvals, void *gmeta,
                                           void *dense_q_out, void *stream)
 {
     if (!ctx || !dY || !gvals || !gmeta) return SSTE_ERR_INVALID_ARG;
     if (gdt != SSTE_BF16 || (odt != SSTE_BF16 && odt != SSTE_E5M2)) return SSTE_ERR_DTYPE;
-    if (odt == SSTE_E5M2 && !gscale_dev) return SSTE_ERR_INVALID_ARG;
+    if (odt == SSTE_E5M2 && !g_amax_dev) return SSTE_ERR_INVALID_ARG;
+    if (counter_cols < 0 || counter_cols > O) return SSTE_ERR_INVALID_ARG;
+    const uint32_t ccols = static_cast<uint32_t>(counter_cols == 0 ? O : counter_cols);
     if (odt == SSTE_BF16 && dense_q_out) return SSTE_ERR_INVALID_ARG;
     if (!sste_mult128(O) || !sste_mult128(T) || (token_offset % 4) != 0) return SSTE_ERR_SHAPE;
     if (!sste_aligned(dY, 128) || !sste_aligned(gvals, 128) || !sste_aligned(gmeta, 128) ||
@@ -775,14 +864,16 @@ extern "C" sste_status sste_mvue_sparsify(sste_ctx *ctx, const void *dY, int T, 
     const dim3 grid(O / 128, T / 128);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const uint32_t key0 = static_cast<uint32_t>(seed), key1 = static_cast<uint32_t>(seed >> 32);
-    if (odt == SSTE_E5M2)
-        sste_launch(mvue_kernel<true>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(dY), O, T,
-                    key0, key1, tensor_id, step, token_offset / 4, gscale_dev, gvals, static_cast<uint8_t *>(gmeta),
-                    dense_q_out);
-    else
-        sste_launch(mvue_kernel<false>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(dY), O, T,
-                    key0, key1, tensor_id, step, token_offset / 4, nullptr, gvals, static_cast<uint8_t *>(gmeta),
-                    nullptr);
+    const uint4 *g = static_cast<const uint4 *>(dY);
+    uint8_t *gm = static_cast<uint8_t *>(gmeta);
+    const uint64_t tg0 = token_offset / 4;
+    const bool f8 = (odt == SSTE_E5M2), any = (ccols % 4) != 0;
+#define SSTE_MVUE_LAUNCH(F8, ANY)                                                                                   \
+    sste_launch(mvue_kernel<F8, ANY>, dim3(grid), dim3(EW_THREADS), 0, s, g, O, T, key0, key1, tensor_id, step, tg0, \
+                ccols, F8 ? g_amax_dev : nullptr, gvals, gm, F8 ? dense_q_out : nullptr)
+    if (f8) { if (any) SSTE_MVUE_LAUNCH(true, true); else SSTE_MVUE_LAUNCH(true, false); }
+    else { if (any) SSTE_MVUE_LAUNCH(false, true); else SSTE_MVUE_LAUNCH(false, false); }
+#undef SSTE_MVUE_LAUNCH
     return launch_result();
 }
 
@@ -830,20 +921,10 @@ extern "C" sste_status sste_fp8_scale(sste_ctx *ctx, const float *amax_dev, sste
     return launch_result();
 }
 
-extern "C" sste_status sste_scalar_mul(sste_ctx *ctx, const float *a_dev, const float *b_dev, float *out_dev,
-                                       void *stream)
-{
-    if (!ctx || !a_dev || !b_dev || !out_dev) return SSTE_ERR_INVALID_ARG;
-    sste_device_guard guard(ctx->device);
-    if (!guard.ok) return SSTE_ERR_CUDA;
-    sste_launch(scalar_mul_kernel, dim3(1), dim3(1), 0, static_cast<cudaStream_t>(stream), a_dev, b_dev, out_dev);
-    return launch_result();
-}
-
-extern "C" sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n, const float *scale_dev,
+extern "C" sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n, const float *amax_dev,
                                          sste_dtype odt, void *q, void *stream)
 {
-    if (!ctx || !x || !scale_dev || !q) return SSTE_ERR_INVALID_ARG;
+    if (!ctx || !x || !amax_dev || !q) return SSTE_ERR_INVALID_ARG;
     if (odt != SSTE_E4M3 && odt != SSTE_E5M2) return SSTE_ERR_DTYPE;
     if (n == 0 || n % 16 != 0) return SSTE_ERR_SHAPE;
     if (!sste_aligned(x, 16) || !sste_aligned(q, 16)) return SSTE_ERR_ALIGN;
@@ -854,10 +935,10 @@ extern "C" sste_status sste_quantize_fp8(sste_ctx *ctx, const void *x, size_t n,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (odt == SSTE_E5M2)
         sste_launch(quantize_kernel<true>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(x),
-                    n_chunks, scale_dev, static_cast<uint2 *>(q));
+                    n_chunks, amax_dev, static_cast<uint2 *>(q));
     else
         sste_launch(quantize_kernel<false>, dim3(grid), dim3(EW_THREADS), 0, s, static_cast<const uint4 *>(x),
-                    n_chunks, scale_dev, static_cast<uint2 *>(q));
+                    n_chunks, amax_dev, static_cast<uint2 *>(q));
     return launch_result();
 }
 
@@ -893,5 +974,58 @@ extern "C" sste_status sste_flip_count(sste_ctx *ctx, const void *meta_prev, con
     SSTE_CUDA_TRY(cudaMemsetAsync(count_dev, 0, sizeof(unsigned long long), s));
     sste_launch(flip_count_kernel, dim3(grid_for(n_vec, ctx->sm_count)), dim3(EW_THREADS), 0, s,
                 static_cast<const uint4 *>(meta_prev), static_cast<const uint4 *>(meta_cur), n_vec, count_dev);
+    return launch_result();
+}
+
+extern "C" sste_status sste_decompress(sste_ctx *ctx, const void *vals, const void *meta, int rows, int k, sste_dtype dt,
+                                       void *dense_out, void *stream)
+{
+    if (!ctx || !vals || !meta || !dense_out) return SSTE_ERR_INVALID_ARG;
+    if (dt != SSTE_BF16 && dt != SSTE_E4M3 && dt != SSTE_E5M2) return SSTE_ERR_DTYPE;
+    if (!sste_mult128(rows) || !sste_mult128(k)) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(vals, 16) || !sste_aligned(meta, 16) || !sste_aligned(dense_out, 16)) return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const bool eight = (dt != SSTE_BF16);
+    const size_t n_units = static_cast<size_t>(rows) * k / (eight ? 32 : 16);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (eight)
+        sste_launch(decompress_kernel<true>, dim3(grid_for(n_units, ctx->sm_count)), dim3(EW_THREADS), 0, s,
+                    static_cast<const uint4 *>(vals), static_cast<const uint8_t *>(meta), k, n_units,
+                    static_cast<uint4 *>(dense_out));
+    else
+        sste_launch(decompress_kernel<false>, dim3(grid_for(n_units, ctx->sm_count)), dim3(EW_THREADS), 0, s,
+                    static_cast<const uint4 *>(vals), static_cast<const uint8_t *>(meta), k, n_units,
+                    static_cast<uint4 *>(dense_out));
+    return launch_result();
+}
+
+extern "C" int sste_padded_dim(int n) { return n <= 0 ? 0 : (n + 127) / 128 * 128; }
+
+extern "C" sste_status sste_pad_2d(sste_ctx *ctx, const void *src, int rows, int cols, void *dst, int rows_p, int cols_p,
+                                   void *stream)
+{
+    if (!ctx || !src || !dst) return SSTE_ERR_INVALID_ARG;
+    if (rows <= 0 || cols <= 0 || rows_p < rows || cols_p < cols || cols_p % 8 != 0) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(src, 2) || !sste_aligned(dst, 16)) return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const size_t n_vec = static_cast<size_t>(rows_p) * cols_p / 8;
+    sste_launch(pad_2d_kernel, dim3(grid_for(n_vec, ctx->sm_count)), dim3(EW_THREADS), 0, static_cast<cudaStream_t>(stream),
+                static_cast<const uint16_t *>(src), rows, cols, static_cast<uint4 *>(dst), cols_p, n_vec);
+    return launch_result();
+}
+
+extern "C" sste_status sste_crop_2d(sste_ctx *ctx, const void *src, int rows_p, int cols_p, void *dst, int rows, int cols,
+                                    void *stream)
+{
+    if (!ctx || !src || !dst) return SSTE_ERR_INVALID_ARG;
+    if (rows <= 0 || cols <= 0 || rows_p < rows || cols_p < cols) return SSTE_ERR_SHAPE;
+    if (!sste_aligned(src, 2) || !sste_aligned(dst, 2)) return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    const size_t n = static_cast<size_t>(rows) * cols;
+    sste_launch(crop_2d_kernel, dim3(grid_for(n, ctx->sm_count)), dim3(EW_THREADS), 0, static_cast<cudaStream_t>(stream),
+                static_cast<const uint16_t *>(src), cols_p, static_cast<uint16_t *>(dst), cols, n);
     return launch_result();
 }

@@ -24,7 +24,6 @@ namespace {
 
 constexpr int BM = 128;            // rows of A per CTA (a pair covers 256)
 constexpr int TMEM_COLS = 512;
-constexpr int META_REGIONS = 8;   // metadata regions of 16 columns (four atoms) after the accumulators
 constexpr int STAGING_BYTES = 32768;   // two epilogue panels of 128 x 64 bf16
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // two seconds of wall time (%globaltimer)
 
@@ -240,9 +239,14 @@ __host__ __device__ constexpr uint32_t instr_desc(bool sparse, uint32_t afmt, ui
 struct GemmParams {
     int M, N, K;            // logical problem: D[M, N] = A[M, K] * B
     void *D;                // output (used by the direct-store fp32 epilogue)
-    const float *out_scale; // device scalar or null
+    // FP8 operands (Sec. 5.2): device scalars max|a|, max|b| of the tensors the operands were quantised from and the
+    // largest finite value of each operand's format; the epilogue multiplies by 1/scale_a * 1/scale_b.  Null for bf16.
+    const float *a_amax, *b_amax;
+    float a_fp8_max, b_fp8_max;
+    unsigned int *out_amax; // nullable: receives max|D| (bit pattern of a non-negative fp32) by atomic maximum
     unsigned int *status;
     uint32_t afmt, bfmt;    // operand format codes of the instruction descriptor
+    const uint8_t *b_vals;  // compressed-B kernels: the 2:4 values of B [K, N/2]; its metadata image is `meta`
     int splits;             // split-K factor of the tiles from `split_from` on (1 = none)
     int split_from;         // first split tile: tiles below it are computed whole
     float *partials;        // split-K: fp32 partial tiles [tile][cta][split][128][BN], summed by splitk_reduce_kernel
@@ -261,7 +265,7 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 // twice the K of one B row); the dense kernel pairs it with one B sub-tile.  A sparse tile of BN = 256
 // leaves room for one accumulator buffer beside the metadata regions in the 512 tensor-memory columns;
 // BN <= 192, and every dense tile, has two, so the epilogue of a tile overlaps the next tile's main loop.
-template <bool SPARSE, int BN>
+template <bool SPARSE, int BN, bool BCOMP = false>
 struct Cfg {
     static constexpr int A_STAGE = 16384;                        // 128 rows x 128 bytes
     static constexpr int B_SUB = (BN / 2) * 128;                 // this CTA's half of one B sub-tile
@@ -269,24 +273,30 @@ struct Cfg {
     static constexpr int STAGE = A_STAGE + B_STAGE;
     static constexpr int FIT = (232448 - 1024 - 512 - STAGING_BYTES) / STAGE;   // 227 KB of shared memory per CTA
     static constexpr int STAGES = FIT > 8 ? 8 : FIT;
-    static constexpr int ACC_BUFS = (!SPARSE || BN <= 192) ? 2 : 1;   // the dense kernel keeps no metadata in TMEM
+    static constexpr int ACC_BUFS = (!SPARSE || BN <= 224) ? 2 : 1;   // the dense kernel keeps no metadata in TMEM
     static constexpr int META_COL0 = ACC_BUFS * BN;              // metadata regions follow the accumulators
-    static constexpr int THREADS = SPARSE ? 320 : 192;           // + 4 metadata warps for the sparse kernels
+    static constexpr int META_FIT = (TMEM_COLS - META_COL0) / 16;
+    static constexpr int META_REGIONS = !SPARSE ? 1 : (META_FIT > 8 ? 8 : META_FIT);   // regions of 16 columns (four atoms)
+    static constexpr int THREADS = (SPARSE || BCOMP) ? 320 : 192;     // + 4 metadata (sparse A) or expander (compressed B) warps
+    static constexpr int PANEL = (BN % 64 == 0) ? 64 : 32;       // columns per epilogue panel (one TMA store)
     static constexpr int SMEM_BYTES = STAGES * STAGE + STAGING_BYTES + 1024 /* alignment slack */ + 512 /* barriers */;
     static_assert(META_COL0 + (SPARSE ? META_REGIONS * 16 : 0) <= TMEM_COLS, "tensor memory budget");
+    static_assert(!SPARSE || META_REGIONS >= 4, "metadata regions");
     static_assert(STAGES >= 3, "pipeline depth");
 };
 
 // ELT: operand element size in bytes (2 = bf16 via kind::f16, 1 = fp8 via kind::f8f6f4).
 // OUT_T: store D transposed (out[n, m]); OUT_F32: fp32 output (direct stores) instead of bf16 (TMA stores).
-template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Cfg<SPARSE, BN>::THREADS, 1)
+// BCOMP: the (dense-product) B operand is given in compressed 2:4 form and expanded in shared memory.
+template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32, bool BCOMP = false>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Cfg<SPARSE, BN, BCOMP>::THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_p,
             const uint8_t *__restrict__ meta, const GemmParams p)
 {
     sste_pdl_trigger();
-    using C = Cfg<SPARSE, BN>;
+    using C = Cfg<SPARSE, BN, BCOMP>;
+    constexpr int META_REGIONS = C::META_REGIONS;
     constexpr int NS = C::STAGES;
     constexpr int NB = C::ACC_BUFS;
     constexpr bool F8 = (ELT == 1);
@@ -296,10 +306,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     constexpr int ATOMS_PER_STAGE = SPARSE ? BK / 128 : 1;   // metadata atoms (128 logical K) per stage
     constexpr int B_CHUNK_N = 128 / ELT;              // MN-major: N elements per 128-byte row
     constexpr int B_CHUNKS_HALF = (BN / 2) / B_CHUNK_N;
-    constexpr uint32_t STAGE_TX = 2u * C::STAGE;      // both CTAs' operand bytes
-    constexpr int PANELS = BN / 64;                   // the epilogue works in panels of 64 columns
-    constexpr int DIRECT_PANELS = PANELS - 2;         // the last two go through registers (early release)
+    constexpr uint32_t STAGE_TX = 2u * (BCOMP ? C::A_STAGE : C::STAGE);   // both CTAs' bytes that arrive by TMA
+    constexpr int PANEL = C::PANEL;                   // the epilogue works in panels of 64 (or 32) columns
+    constexpr int DIRECT_PANELS = (BN - 128) / PANEL; // the last 128 columns go through registers (early release)
     static_assert(BMAJ == BMajor::K || (BN / 2) % B_CHUNK_N == 0, "MN-major B needs whole 128-byte chunks per CTA");
+    static_assert(PANEL == 64 || (OUT_T && !OUT_F32), "32-column panels exist for the transposed bf16 store only");
+    static_assert(!BCOMP || (!SPARSE && BMAJ == BMajor::MN), "compressed B: dense A, MN-major B");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -317,7 +329,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     volatile uint32_t *tmem_slot_ptr = reinterpret_cast<volatile uint32_t *>(bars_generic + 8u * MISC);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_generic + 8u * (MISC + 1));
     uint8_t *staging_generic = smem_raw + (staging - smem_u32(smem_raw));
-    static_assert(8 * (MISC + 2) <= 512, "barrier block");
+    static_assert(8 * (MISC + 2) + 64 <= 512, "barrier block (+ the expander's 16-entry selector table)");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -346,13 +358,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int k_atoms = p.K / 128;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        // full: the producer's arrival with the TMA byte count (+ the eight expander warps of the pair)
+        for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), BCOMP ? 9 : 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 2); }
         for (int r = 0; r < META_REGIONS; ++r) { mbar_init(meta_full_bar(r), 8); mbar_init(meta_empty_bar(r), 1); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_a);
-        prefetch_tensormap(&map_b);
+        if (!BCOMP) prefetch_tensormap(&map_b);
         if (!OUT_F32) prefetch_tensormap(&map_d);
     }
     if (warp == 1) {
@@ -387,7 +400,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint32_t b_dst = a_dst + C::A_STAGE;
                     // A: 128 bytes per row = BK/2 compressed (sparse) or BK dense elements
                     tma_load_2d(a_dst, &map_a, lead_full, kb * (SPARSE ? BK / 2 : BK), m0);
-                    if (BMAJ == BMajor::K) {
+                    if (BCOMP) {
+                        // B is written into the stage by the expander warps
+                    } else if (BMAJ == BMajor::K) {
 #pragma unroll
                         for (int u = 0; u < B_SUBS; ++u)
                             tma_load_2d(b_dst + u * C::B_SUB, &map_b, lead_full, kb * BK + u * SUB_K, n0);
@@ -470,7 +485,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
         const int quarter = warp & 3;                  // tensor-memory lanes [32*quarter, 32*quarter + 32)
         const int row = quarter * 32 + lane;           // row of this CTA's 128 x BN accumulator
-        const float scale = p.out_scale ? *p.out_scale : 1.0f;
+        const float scale = sste_out_scale(p.a_amax, p.a_fp8_max, p.b_amax, p.b_fp8_max);
+        const bool want_amax = (p.out_amax != nullptr);
+        uint32_t amax2 = 0;                            // bf16 output: running max of the magnitude bits, two lanes of 16
+        float amaxf = 0.0f;                            // fp32 output
         const bool store_thread = (threadIdx.x == 64);
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         uint32_t local_tile = 0, panel_it = 0;
@@ -494,20 +512,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     tmem_ld_wait();
                     const int m = m0 + row;
                     if (m < p.M && n0 + c0 < p.N) {
+                        float v[32];
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) v[c] = __fmul_rn(__uint_as_float(r[c]), scale);
+                        if (want_amax) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) amaxf = fmaxf(amaxf, fabsf(v[c]));
+                        }
                         if (OUT_T) {
                             float *out = static_cast<float *>(p.D);
 #pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                out[static_cast<size_t>(n0 + c0 + c) * p.M + m] = __fmul_rn(__uint_as_float(r[c]), scale);
+                            for (int c = 0; c < 32; ++c) out[static_cast<size_t>(n0 + c0 + c) * p.M + m] = v[c];
                         } else {
                             float4 *out = reinterpret_cast<float4 *>(static_cast<float *>(p.D) +
                                                                      static_cast<size_t>(m) * p.N + n0 + c0);
 #pragma unroll
-                            for (int c = 0; c < 8; ++c)
-                                out[c] = make_float4(__fmul_rn(__uint_as_float(r[4 * c]), scale),
-                                                     __fmul_rn(__uint_as_float(r[4 * c + 1]), scale),
-                                                     __fmul_rn(__uint_as_float(r[4 * c + 2]), scale),
-                                                     __fmul_rn(__uint_as_float(r[4 * c + 3]), scale));
+                            for (int c = 0; c < 8; ++c) out[c] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
                         }
                     }
                 }
@@ -548,16 +568,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (store_thread) mbar_arrive_cluster(lead_acc_empty);
                 continue;
             }
-            // bf16 output in panels of 64 columns through two 16 KB staging buffers and TMA stores.
+            // bf16 output in panels of PANEL columns through two 16 KB staging buffers and TMA stores.
             // 32 accumulator columns -> bf16 -> staging buffer `sb`, columns [c0, c0 + 32) of the panel
             auto stage_chunk = [&](const uint32_t (&r)[32], uint8_t *sb, int c0) {
                 if (OUT_T) {
-                    // staging[n][m]: 64 rows of 128 bf16; a warp writes 32 consecutive m per n
+                    // staging[n][m]: PANEL rows of 128 bf16; a warp writes 32 consecutive m per n
                     uint16_t *st = reinterpret_cast<uint16_t *>(sb);
 #pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        st[(c0 + c) * BM + row] =
-                            static_cast<uint16_t>(sste_f32_to_bf16_bits(__fmul_rn(__uint_as_float(r[c]), scale)));
+                    for (int c = 0; c < 32; c += 2) {
+                        const uint32_t lo = sste_f32_to_bf16_bits(__fmul_rn(__uint_as_float(r[c]), scale));
+                        const uint32_t hi = sste_f32_to_bf16_bits(__fmul_rn(__uint_as_float(r[c + 1]), scale));
+                        st[(c0 + c) * BM + row] = static_cast<uint16_t>(lo);
+                        st[(c0 + c + 1) * BM + row] = static_cast<uint16_t>(hi);
+                        if (want_amax) amax2 = __vmaxu2(amax2, (lo | (hi << 16)) & 0x7fff7fffu);
+                    }
                 } else {
                     // [128 rows][64 bf16] with the 128-byte swizzle of the TMA store: 16-byte chunk index ^= row & 7
                     uint8_t *dst = sb + row * 128;
@@ -570,6 +594,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                             const float lo = __fmul_rn(__uint_as_float(r[8 * c + 2 * e]), scale);
                             const float hi = __fmul_rn(__uint_as_float(r[8 * c + 2 * e + 1]), scale);
                             w[e] = sste_f32_to_bf16_bits(lo) | (sste_f32_to_bf16_bits(hi) << 16);
+                            if (want_amax) amax2 = __vmaxu2(amax2, w[e] & 0x7fff7fffu);
                         }
                         *reinterpret_cast<uint4 *>(dst + (((chunk0 + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
@@ -585,8 +610,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 fence_proxy_async();
                 epilogue_barrier();
                 if (store_thread) {
-                    if (OUT_T) tma_store_2d(&map_d, staging + off, m0, n0 + 64 * panel);
-                    else tma_store_2d(&map_d, staging + off, n0 + 64 * panel, m0);
+                    if (OUT_T) tma_store_2d(&map_d, staging + off, m0, n0 + PANEL * panel);
+                    else tma_store_2d(&map_d, staging + off, n0 + PANEL * panel, m0);
                     tma_store_commit();
                 }
                 ++panel_it;
@@ -595,34 +620,51 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             for (int pnl = 0; pnl < DIRECT_PANELS; ++pnl) {
                 const uint32_t off = acquire_staging();
                 uint32_t ra[32], rb[32];
-                tmem_ld_32x32(acc_base + 64 * pnl, ra);
-                tmem_ld_32x32(acc_base + 64 * pnl + 32, rb);
+                tmem_ld_32x32(acc_base + PANEL * pnl, ra);
+                if (PANEL == 64) tmem_ld_32x32(acc_base + PANEL * pnl + 32, rb);
                 tmem_ld_wait();
                 stage_chunk(ra, staging_generic + off, 0);
-                stage_chunk(rb, staging_generic + off, 32);
+                if (PANEL == 64) stage_chunk(rb, staging_generic + off, 32);
                 store_panel(off, pnl);
             }
-            // last two panels -> registers, then the accumulator buffer is free for the next tile
+            // last 128 columns -> registers, then the accumulator buffer is free for the next tile
             uint32_t r0[32], r1[32], r2[32], r3[32];
-            tmem_ld_32x32(acc_base + 64 * DIRECT_PANELS, r0);
-            tmem_ld_32x32(acc_base + 64 * DIRECT_PANELS + 32, r1);
-            tmem_ld_32x32(acc_base + 64 * DIRECT_PANELS + 64, r2);
-            tmem_ld_32x32(acc_base + 64 * DIRECT_PANELS + 96, r3);
+            tmem_ld_32x32(acc_base + BN - 128, r0);
+            tmem_ld_32x32(acc_base + BN - 96, r1);
+            tmem_ld_32x32(acc_base + BN - 64, r2);
+            tmem_ld_32x32(acc_base + BN - 32, r3);
             tmem_ld_wait();
             tc_fence_before();
             {
                 const uint32_t off = acquire_staging();      // includes the barrier after everyone's loads
                 if (store_thread) mbar_arrive_cluster(lead_acc_empty);
                 stage_chunk(r0, staging_generic + off, 0);
-                stage_chunk(r1, staging_generic + off, 32);
+                if (PANEL == 64) stage_chunk(r1, staging_generic + off, 32);
                 store_panel(off, DIRECT_PANELS);
+            }
+            if (PANEL == 32) {
+                const uint32_t off = acquire_staging();
+                stage_chunk(r1, staging_generic + off, 0);
+                store_panel(off, DIRECT_PANELS + 1);
             }
             {
                 const uint32_t off = acquire_staging();
                 stage_chunk(r2, staging_generic + off, 0);
-                stage_chunk(r3, staging_generic + off, 32);
-                store_panel(off, DIRECT_PANELS + 1);
+                if (PANEL == 64) stage_chunk(r3, staging_generic + off, 32);
+                store_panel(off, DIRECT_PANELS + (PANEL == 64 ? 1 : 2));
             }
+            if (PANEL == 32) {
+                const uint32_t off = acquire_staging();
+                stage_chunk(r3, staging_generic + off, 0);
+                store_panel(off, DIRECT_PANELS + 3);
+            }
+        }
+        if (want_amax) {
+            // max|D| of this warp's share, as the bits of a non-negative fp32 (they order like unsigned integers)
+            uint32_t best = OUT_F32 ? __float_as_uint(amaxf) : (max(amax2 & 0xffffu, amax2 >> 16) << 16);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+            if (lane == 0 && best != 0) atomicMax(p.out_amax, best);
         }
         if (store_thread && !OUT_F32) tma_store_wait_all();
     } else if (SPARSE) {
@@ -681,6 +723,110 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             h1 = h2;
             h2 = l_issue(q2);
         }
+    } else if (BCOMP) {
+        // ------------------------------------------------------------ expander warps (6..9, both CTAs)
+        // grad_X = grad_Z S(W) reads S(W) [O, I] as its MN-major B operand.  Here S(W) is given as the forward's
+        // compressed operand (2:4 values + metadata image) and every stage's K rows are expanded into the shared-
+        // memory image a TMA load of the dense matrix would have left: rows of 128 bytes of N, 16-byte chunks
+        // XOR-swizzled with the row, +0 in the pruned positions.  A unit is 16 bytes of values (8 groups of fp8,
+        // 4 of bf16) = 32 bytes of the dense row; the loads of the next stage are in flight while this one is
+        // expanded.
+        constexpr int SEGS = (BN / 2) * ELT / 32;          // units per K row of this CTA's half of the tile
+        constexpr int UNITS = BK * SEGS / 128;             // units per thread and stage
+        static_assert(!BCOMP || (BK * SEGS) % 128 == 0, "units per stage");
+        const int t = static_cast<int>(threadIdx.x) - 192;
+        // byte-permute selectors per metadata nibble p0 | p1 << 2: which source byte feeds each output byte
+        // (4 = a zero byte).  bf16: low / high 16 bits select the two output words of a group from the pair word;
+        // fp8: 16 bits select the output word of a group from its two value bytes (0, 1).
+        uint32_t *lut = reinterpret_cast<uint32_t *>(bars_generic + 8u * (MISC + 2));
+        if (t < 16) {
+            const uint32_t p0 = t & 3, p1 = t >> 2;
+            uint32_t sel = 0;
+            for (uint32_t h = 0; h < 4; ++h) {
+                if (F8) sel |= (h == p0 ? 0u : h == p1 ? 1u : 4u) << (4 * h);
+                else sel |= (h == p0 ? 0x10u : h == p1 ? 0x32u : 0x44u) << (8 * h);
+            }
+            lut[t] = sel;
+        }
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        const int n_half_vals = p.N / 2;                   // compressed values per row of B
+        const int n_atoms = p.N / 128;
+        int e_unit = pair, e_kb = 0, e_kend = 0, e_n0 = 0;
+        auto e_setup = [&]() {
+            if (e_unit >= num_units) return;
+            const Unit u = decode(e_unit);
+            e_n0 = (u.tile / m_tiles) * BN + static_cast<int>(rank) * (BN / 2);
+            e_kb = u.split * u.k_blocks;
+            e_kend = e_kb + u.k_blocks;
+        };
+        auto e_issue = [&](uint4 (&v)[UNITS], uint32_t (&m)[UNITS]) -> bool {
+            if (e_unit >= num_units) return false;
+#pragma unroll
+            for (int j = 0; j < UNITS; ++j) {
+                const int un = j * 128 + t;
+                const uint32_t krow = static_cast<uint32_t>(e_kb * BK + un / SEGS);
+                const uint32_t ncol = static_cast<uint32_t>(e_n0 + (un % SEGS) * (32 / ELT));
+                if (ncol < static_cast<uint32_t>(p.N) && krow < static_cast<uint32_t>(p.K)) {
+                    v[j] = __ldg(reinterpret_cast<const uint4 *>(
+                        p.b_vals + (static_cast<size_t>(krow) * n_half_vals + ncol / 2) * ELT));
+                    const uint8_t *atom = meta + (static_cast<size_t>(krow >> 7) * n_atoms + (ncol >> 7)) * 2048;
+                    if (F8) m[j] = __ldg(reinterpret_cast<const uint32_t *>(atom + sste_meta_atom_byte8(krow & 127u, ncol & 127u)));
+                    else m[j] = __ldg(reinterpret_cast<const uint16_t *>(atom + sste_meta_atom_byte16(krow & 127u, ncol & 127u)));
+                } else {
+                    v[j] = make_uint4(0, 0, 0, 0);
+                    m[j] = 0x44444444u;                    // any valid code: the values are zero
+                }
+            }
+            if (++e_kb >= e_kend) {
+                e_unit += num_pairs;
+                e_setup();
+            }
+            return true;
+        };
+        e_setup();
+        uint4 cv[UNITS], nv[UNITS];
+        uint32_t cm[UNITS], nm[UNITS];
+        bool have = e_issue(cv, cm);
+        uint32_t it = 0;
+        while (have) {
+            const bool have_next = e_issue(nv, nm);
+            const int s = it % NS;
+            const uint32_t ph = (it / NS) & 1u;
+            if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, p.status, abort_flag)) break;
+            uint8_t *b_dst = smem_raw + (smem_base - smem_u32(smem_raw)) + s * C::STAGE + C::A_STAGE;
+#pragma unroll
+            for (int j = 0; j < UNITS; ++j) {
+                const int un = j * 128 + t;
+                const int r = un / SEGS, seg = un % SEGS;
+                const uint32_t w[4] = {cv[j].x, cv[j].y, cv[j].z, cv[j].w};
+                uint32_t o[8];
+                if (F8) {
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        const uint32_t pairw = (g & 1) ? (w[g >> 1] >> 16) : w[g >> 1];    // value bytes 0, 1
+                        o[g] = __byte_perm(pairw, 0, lut[(cm[j] >> (4 * g)) & 0xfu]);
+                    }
+                } else {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const uint32_t sel = lut[(cm[j] >> (4 * g)) & 0xfu];
+                        o[2 * g] = __byte_perm(w[g], 0, sel & 0xffffu);
+                        o[2 * g + 1] = __byte_perm(w[g], 0, sel >> 16);
+                    }
+                }
+                uint8_t *rowp = b_dst + (seg >> 2) * (BK * 128) + r * 128;
+                const int j0 = (seg & 3) * 2;
+                *reinterpret_cast<uint4 *>(rowp + ((j0 ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4 *>(rowp + (((j0 + 1) ^ (r & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+            fence_proxy_async();        // the tensor core reads the stage through the async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(full_bar(s), 0));
+#pragma unroll
+            for (int j = 0; j < UNITS; ++j) { cv[j] = nv[j]; cm[j] = nm[j]; }
+            have = have_next;
+            ++it;
+        }
     }
 
     // ---------------------------------------------------------------- teardown
@@ -719,13 +865,16 @@ bool make_map(const sste_ctx *ctx, CUtensorMap *map, const void *base, int elt, 
 // the fp32 partial tiles [split tile][cta][split][128][bn]).  One thread per 8 consecutive n.
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, int splits, int m_tiles, int split_from,
-                     int n_split_tiles, const float *__restrict__ out_scale, uint4 *__restrict__ out)
+                     int n_split_tiles, const float *__restrict__ a_amax, float a_fp8_max,
+                     const float *__restrict__ b_amax, float b_fp8_max, unsigned int *__restrict__ out_amax,
+                     uint4 *__restrict__ out)
 {
     sste_pdl_trigger();
     const int vec_per_row = bn / 8;
     const size_t vecs = static_cast<size_t>(n_split_tiles) * 2 * BM * vec_per_row;
     sste_pdl_wait();
-    const float scale = out_scale ? *out_scale : 1.0f;
+    const float scale = sste_out_scale(a_amax, a_fp8_max, b_amax, b_fp8_max);
+    uint32_t amax2 = 0;
     for (size_t v = static_cast<size_t>(blockIdx.x) * 256 + threadIdx.x; v < vecs; v += static_cast<size_t>(gridDim.x) * 256) {
         const int col = static_cast<int>(v % vec_per_row) * 8;
         const int row = static_cast<int>((v / vec_per_row) % BM);
@@ -746,7 +895,17 @@ splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, i
 #pragma unroll
         for (int e = 0; e < 4; ++e)
             w[e] = sste_f32_to_bf16_bits(__fmul_rn(acc[2 * e], scale)) | (sste_f32_to_bf16_bits(__fmul_rn(acc[2 * e + 1], scale)) << 16);
+        if (out_amax) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) amax2 = __vmaxu2(amax2, w[e] & 0x7fff7fffu);
+        }
         out[(static_cast<size_t>(m) * N + n) / 8] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    if (out_amax) {
+        uint32_t best = max(amax2 & 0xffffu, amax2 >> 16) << 16;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+        if ((threadIdx.x & 31) == 0 && best != 0) atomicMax(out_amax, best);
     }
 }
 
@@ -768,11 +927,11 @@ struct DeviceOnce {
 struct SplitPlan { int splits, split_from; };
 SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn);
 
-template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32>
+template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32, bool BCOMP = false>
 sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void *meta, const GemmParams &p,
                    cudaStream_t stream)
 {
-    using C = Cfg<SPARSE, BN>;
+    using C = Cfg<SPARSE, BN, BCOMP>;
     constexpr int BK = (SPARSE ? 256 : 128) / ELT;
     CUtensorMap map_a, map_b, map_d, map_p;
     bool ok;
@@ -780,19 +939,21 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         ok = make_map(ctx, &map_a, A, ELT, p.M, p.K / 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_128B);
     else
         ok = make_map(ctx, &map_a, A, ELT, p.M, p.K, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B);
-    if (BMAJ == BMajor::K)   // B stored [N, K]: sub-tiles of BN/2 rows by 128 bytes of K
+    if (BCOMP)               // B is expanded from its compressed form by the kernel: no map
+        map_b = map_a;
+    else if (BMAJ == BMajor::K)   // B stored [N, K]: sub-tiles of BN/2 rows by 128 bytes of K
         ok = ok && make_map(ctx, &map_b, B, ELT, p.N, p.K, 128 / ELT, BN / 2, CU_TENSOR_MAP_SWIZZLE_128B);
     else                     // B stored [K, N]: chunks of 128 bytes of N by BK rows of K
         ok = ok && make_map(ctx, &map_b, B, ELT, p.K, p.N, 128 / ELT, BK, CU_TENSOR_MAP_SWIZZLE_128B);
     if (OUT_F32) {
         map_d = map_a;       // unused: the fp32 epilogue stores directly
-    } else if (OUT_T) {      // out[N, M] bf16: panels of 128 m x 64 n
-        ok = ok && make_map(ctx, &map_d, p.D, 2, p.N, p.M, BM, 64, CU_TENSOR_MAP_SWIZZLE_NONE);
+    } else if (OUT_T) {      // out[N, M] bf16: panels of 128 m x 64 (or 32) n
+        ok = ok && make_map(ctx, &map_d, p.D, 2, p.N, p.M, BM, C::PANEL, CU_TENSOR_MAP_SWIZZLE_NONE);
     } else {                 // out[M, N] bf16: panels of 64 n x 128 m, 128-byte swizzle
         ok = ok && make_map(ctx, &map_d, p.D, 2, p.M, p.N, 64, BM, CU_TENSOR_MAP_SWIZZLE_128B);
     }
     if (!ok) return SSTE_ERR_CUDA;
-    auto kern = gemm_kernel<SPARSE, BMAJ, ELT, BN, OUT_T, OUT_F32>;
+    auto kern = gemm_kernel<SPARSE, BMAJ, ELT, BN, OUT_T, OUT_F32, BCOMP>;
     // The opt-in to more than 48 KB of dynamic shared memory is a per-DEVICE attribute of the kernel:
     // set once per (instantiation, device), under a lock (contexts may be used from several host threads).
     static DeviceOnce attr_done;
@@ -802,6 +963,8 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         return SSTE_ERR_CUDA;
     const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM), n_tiles = (p.N + BN - 1) / BN;
     GemmParams pp = p;
+    if (BCOMP) pp.b_vals = static_cast<const uint8_t *>(B);
+    if (pp.out_amax && cudaMemsetAsync(pp.out_amax, 0, sizeof(unsigned int), stream) != cudaSuccess) return SSTE_ERR_CUDA;
     const int tiles = m_tiles * n_tiles;
     SplitPlan plan{1, tiles};
     if (!OUT_F32 && !OUT_T) plan = pick_split_plan(ctx, tiles, (p.K + BK - 1) / BK, SPARSE ? 4 / (BK / 128) : 1, BN);
@@ -824,8 +987,8 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         size_t blocks = (vecs + 255) / 256;
         if (blocks > static_cast<size_t>(ctx->sm_count) * 16) blocks = static_cast<size_t>(ctx->sm_count) * 16;
         if (sste_launch(splitk_reduce_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(256), 0, stream,
-                        pp.partials, p.M, p.N, BN, pp.splits, m_tiles, pp.split_from, n_split_tiles, p.out_scale,
-                        static_cast<uint4 *>(p.D)) != cudaSuccess)
+                        pp.partials, p.M, p.N, BN, pp.splits, m_tiles, pp.split_from, n_split_tiles, p.a_amax,
+                        p.a_fp8_max, p.b_amax, p.b_fp8_max, pp.out_amax, static_cast<uint4 *>(p.D)) != cudaSuccess)
             return SSTE_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return SSTE_ERR_CUDA;
@@ -898,13 +1061,17 @@ sste_status launch_out(const sste_ctx *ctx, const void *A, const void *B, const 
     if (odt == SSTE_F32) return launch<SPARSE, BMAJ, ELT, 256, OUT_T, true>(ctx, A, B, meta, p, s);
     if (odt != SSTE_BF16) return SSTE_ERR_DTYPE;
     constexpr bool MN = (BMAJ == BMajor::MN);
-    int cands[3], n = 0;
+    int cands[4], n = 0;
     cands[n++] = 256;
     if (!(MN && ELT == 1)) cands[n++] = 128;   // MN-major B: each CTA needs whole 128-byte chunks of N
     if (!MN) cands[n++] = 192;
+    if (!MN && SPARSE && OUT_T) cands[n++] = 224;
     int bn = pick_bn(!MN, p.M, p.N, p.K, ctx->sm_count / 2);
     for (int i = 0; i < n; ++i)
         if (cands[i] == g_force_bn) bn = g_force_bn;
+    if constexpr (!MN && SPARSE && OUT_T) {
+        if (bn == 224) return launch<SPARSE, BMAJ, ELT, 224, OUT_T, false>(ctx, A, B, meta, p, s);
+    }
     if constexpr (!MN) {
         if (bn == 192) return launch<SPARSE, BMAJ, ELT, 192, OUT_T, false>(ctx, A, B, meta, p, s);
     }
@@ -912,6 +1079,12 @@ sste_status launch_out(const sste_ctx *ctx, const void *A, const void *B, const 
         if (bn == 128) return launch<SPARSE, BMAJ, ELT, 128, OUT_T, false>(ctx, A, B, meta, p, s);
     }
     return launch<SPARSE, BMAJ, ELT, 256, OUT_T, false>(ctx, A, B, meta, p, s);
+}
+
+// FP8 operands come with the amax of the tensors they were quantised from (both or neither); bf16 with none.
+bool amax_args_ok(int elt, const float *a_amax, const float *b_amax)
+{
+    return elt == 1 ? (a_amax && b_amax) : (!a_amax && !b_amax);
 }
 
 }  // namespace
@@ -924,27 +1097,29 @@ extern "C" sste_status sste_debug_force_splits(int splits)
 }
 extern "C" sste_status sste_debug_force_tile_width(int bn)
 {
-    if (bn != 0 && bn != 128 && bn != 192 && bn != 256) return SSTE_ERR_INVALID_ARG;
+    if (bn != 0 && bn != 128 && bn != 192 && bn != 224 && bn != 256) return SSTE_ERR_INVALID_ARG;
     g_force_bn = bn;
     return SSTE_OK;
 }
 
 extern "C" sste_status sste_linear_fwd(sste_ctx *ctx, const void *X, int T, const void *vals, const void *meta, int O,
-                                       int I, sste_dtype opdt, const float *out_scale_dev, void *Y, sste_dtype ydt,
-                                       void *stream)
+                                       int I, sste_dtype opdt, const float *x_amax_dev, const float *w_amax_dev,
+                                       void *Y, sste_dtype ydt, float *y_amax_out_dev, void *stream)
 {
     if (!ctx || !X || !vals || !meta || !Y) return SSTE_ERR_INVALID_ARG;
     int elt;
     uint32_t code;
     if (!fmt_code(opdt, &elt, &code) || opdt == SSTE_E5M2) return SSTE_ERR_DTYPE;
     if (ydt != SSTE_BF16 && ydt != SSTE_F32) return SSTE_ERR_DTYPE;
+    if (!amax_args_ok(elt, w_amax_dev, x_amax_dev)) return SSTE_ERR_INVALID_ARG;
     if (!sste_mult128(T) || !sste_mult128(O) || !sste_mult128(I)) return SSTE_ERR_SHAPE;
     if (!sste_aligned(X, 128) || !sste_aligned(vals, 128) || !sste_aligned(meta, 128) || !sste_aligned(Y, 128))
         return SSTE_ERR_ALIGN;
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
     // Z^T[O, T] = S(W)[O, I] X^T: M = O, N = T, K = I; the output is stored transposed as Y[T, O]
-    GemmParams p{O, T, I, Y, out_scale_dev, ctx->status_dev, code, code};
+    GemmParams p{O, T, I, Y, w_amax_dev, x_amax_dev, sste_fp8_max(opdt), sste_fp8_max(opdt),
+                 reinterpret_cast<unsigned int *>(y_amax_out_dev), ctx->status_dev, code, code, nullptr};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (elt == 2) return launch_out<true, BMajor::K, 2, true>(ctx, vals, X, meta, p, ydt, s);
     return launch_out<true, BMajor::K, 1, true>(ctx, vals, X, meta, p, ydt, s);
@@ -952,7 +1127,8 @@ extern "C" sste_status sste_linear_fwd(sste_ctx *ctx, const void *X, int T, cons
 
 extern "C" sste_status sste_linear_bwd_weight(sste_ctx *ctx, const void *gvals, const void *gmeta, int O, int T,
                                               sste_dtype gdt, const void *X, int I, sste_dtype xdt,
-                                              const float *out_scale_dev, void *dW, sste_dtype dwdt, void *stream)
+                                              const float *g_amax_dev, const float *x_amax_dev, void *dW,
+                                              sste_dtype dwdt, void *stream)
 {
     if (!ctx || !gvals || !gmeta || !X || !dW) return SSTE_ERR_INVALID_ARG;
     int ea, eb;
@@ -960,35 +1136,52 @@ extern "C" sste_status sste_linear_bwd_weight(sste_ctx *ctx, const void *gvals, 
     if (!fmt_code(gdt, &ea, &ca) || !fmt_code(xdt, &eb, &cb) || ea != eb) return SSTE_ERR_DTYPE;
     if (gdt == SSTE_E4M3 || xdt == SSTE_E5M2) return SSTE_ERR_DTYPE;
     if (dwdt != SSTE_BF16 && dwdt != SSTE_F32) return SSTE_ERR_DTYPE;
+    if (!amax_args_ok(ea, g_amax_dev, x_amax_dev)) return SSTE_ERR_INVALID_ARG;
     if (!sste_mult128(T) || !sste_mult128(O) || !sste_mult128(I)) return SSTE_ERR_SHAPE;
     if (!sste_aligned(X, 128) || !sste_aligned(gvals, 128) || !sste_aligned(gmeta, 128) || !sste_aligned(dW, 128))
         return SSTE_ERR_ALIGN;
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
     // grad_W[O, I] = G[O, T] X[T, I]: M = O, N = I, K = T; X is [K, N] row-major = MN-major B
-    GemmParams p{O, I, T, dW, out_scale_dev, ctx->status_dev, ca, cb};
+    GemmParams p{O, I, T, dW, g_amax_dev, x_amax_dev, sste_fp8_max(gdt), sste_fp8_max(xdt), nullptr,
+                 ctx->status_dev, ca, cb, nullptr};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (ea == 2) return launch_out<true, BMajor::MN, 2, false>(ctx, gvals, X, gmeta, p, dwdt, s);
     return launch_out<true, BMajor::MN, 1, false>(ctx, gvals, X, gmeta, p, dwdt, s);
 }
 
 extern "C" sste_status sste_linear_bwd_input(sste_ctx *ctx, const void *dY, int T, int O, sste_dtype gdt,
-                                             const void *Wt_dense, int I, sste_dtype wdt,
-                                             const float *out_scale_dev, void *dX, sste_dtype xdt, void *stream)
+                                             const void *Wt_dense, const void *vals, const void *meta, int I,
+                                             sste_dtype wdt, const float *g_amax_dev, const float *w_amax_dev,
+                                             void *dX, sste_dtype xdt, float *dx_amax_out_dev, void *stream)
 {
-    if (!ctx || !dY || !Wt_dense || !dX) return SSTE_ERR_INVALID_ARG;
+    if (!ctx || !dY || !dX) return SSTE_ERR_INVALID_ARG;
+    if (!Wt_dense && !(vals && meta)) return SSTE_ERR_INVALID_ARG;
     int ea, eb;
     uint32_t ca, cb;
     if (!fmt_code(gdt, &ea, &ca) || !fmt_code(wdt, &eb, &cb) || ea != eb) return SSTE_ERR_DTYPE;
     if (gdt == SSTE_E4M3 || wdt == SSTE_E5M2) return SSTE_ERR_DTYPE;
     if (xdt != SSTE_BF16 && xdt != SSTE_F32) return SSTE_ERR_DTYPE;
+    if (!amax_args_ok(ea, g_amax_dev, w_amax_dev)) return SSTE_ERR_INVALID_ARG;
     if (!sste_mult128(T) || !sste_mult128(O) || !sste_mult128(I)) return SSTE_ERR_SHAPE;
-    if (!sste_aligned(dY, 128) || !sste_aligned(Wt_dense, 128) || !sste_aligned(dX, 128)) return SSTE_ERR_ALIGN;
+    if (!sste_aligned(dY, 128) || !sste_aligned(Wt_dense, 128) || !sste_aligned(vals, 128) || !sste_aligned(meta, 128) ||
+        !sste_aligned(dX, 128))
+        return SSTE_ERR_ALIGN;
     sste_device_guard guard(ctx->device);
     if (!guard.ok) return SSTE_ERR_CUDA;
     // grad_X[T, I] = grad_Z[T, O] S(W)[O, I]: M = T, N = I, K = O; S(W) is [K, N] row-major = MN-major B
-    GemmParams p{T, I, O, dX, out_scale_dev, ctx->status_dev, ca, cb};
+    GemmParams p{T, I, O, dX, g_amax_dev, w_amax_dev, sste_fp8_max(gdt), sste_fp8_max(wdt),
+                 reinterpret_cast<unsigned int *>(dx_amax_out_dev), ctx->status_dev, ca, cb, nullptr};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!Wt_dense) {
+        // S(W) from the forward's compressed operand, expanded in shared memory (256-wide tiles)
+        const bool f32 = (xdt == SSTE_F32);
+        if (ea == 2)
+            return f32 ? launch<false, BMajor::MN, 2, 256, false, true, true>(ctx, dY, vals, meta, p, s)
+                       : launch<false, BMajor::MN, 2, 256, false, false, true>(ctx, dY, vals, meta, p, s);
+        return f32 ? launch<false, BMajor::MN, 1, 256, false, true, true>(ctx, dY, vals, meta, p, s)
+                   : launch<false, BMajor::MN, 1, 256, false, false, true>(ctx, dY, vals, meta, p, s);
+    }
     if (ea == 2) return launch_out<false, BMajor::MN, 2, false>(ctx, dY, Wt_dense, nullptr, p, xdt, s);
     return launch_out<false, BMajor::MN, 1, false>(ctx, dY, Wt_dense, nullptr, p, xdt, s);
 }

@@ -16,16 +16,21 @@ class SsteLinear:
     """W[O, I] dense master weight (bf16); forward Y = X S(W)^T, backward (dX, dW).
 
     ``fp8=True`` selects the whole-process FP8 variant (Sec. 5.2): E4M3 forward
-    operands, E5M2 output gradient, per-tensor scale = fp8_max / amax computed
-    just in time on the device.  ``track_flips=True`` keeps the previous iteration's
-    metadata and counts the mask entries that changed at every prune (flip rate, Sec. 3.1).
+    operands, E5M2 output gradient, per-tensor scale = fp8_max / amax; the state of a
+    quantised tensor is its amax (one device float), from which every consumer forms the
+    scale itself.  ``dense_copy=True`` also keeps w~ as a dense [O, I] tensor and feeds
+    grad_X from it; by default grad_X expands the compressed operand inside the product.
+    ``track_flips=True`` keeps the previous iteration's metadata and counts the mask entries
+    that changed at every prune (flip rate, Sec. 3.1).
     """
 
     def __init__(self, ctx: B.Context, W: torch.Tensor, T: int, tensor_id: int = 0, seed: int = 0,
-                 fp8: bool = False, out_dtype: torch.dtype = torch.bfloat16, track_flips: bool = False):
+                 fp8: bool = False, out_dtype: torch.dtype = torch.bfloat16, track_flips: bool = False,
+                 dense_copy: bool = False, counter_cols: int = 0):
         assert W.dtype == torch.bfloat16 and W.is_cuda
         self.ctx, self.W, self.T, self.tensor_id, self.seed, self.fp8 = ctx, W, T, tensor_id, seed, fp8
         self.O, self.I = W.shape
+        self.counter_cols = counter_cols
         O, I, dev = self.O, self.I, W.device
         f32 = dict(dtype=torch.float32, device=dev)
         self.beta = torch.zeros(1, **f32)
@@ -33,7 +38,7 @@ class SsteLinear:
         wdt = B.E4M3 if fp8 else B.BF16
         gdt = B.E5M2 if fp8 else B.BF16
         self.vals, self.meta = ctx.alloc_compressed(O, I, wdt)
-        self.w_dense = torch.empty((O, I), dtype=B._TORCH_DT[wdt], device=dev)
+        self.w_dense = torch.empty((O, I), dtype=B._TORCH_DT[wdt], device=dev) if dense_copy else None
         self.gvals, self.gmeta = ctx.alloc_compressed(O, T, gdt)
         self.Y = torch.empty((T, O), dtype=out_dtype, device=dev)
         self.dX = torch.empty((T, I), dtype=out_dtype, device=dev)
@@ -44,15 +49,13 @@ class SsteLinear:
             self.meta_prev = torch.empty_like(self.meta)
             self.flips = torch.zeros(1, dtype=torch.int64, device=dev)   # mask entries changed by the last prune
             self._have_prev = False
+        self.amax = torch.zeros(3, **f32) if fp8 else None     # max|X|, max|w~| (bf16 projection), max|dY|
         if fp8:
-            self.amax = torch.zeros(3, **f32)          # X, w~ (through W and beta), dY
-            self.scale = torch.ones(3, **f32)
-            self.inv = torch.ones(3, **f32)
-            self.inv_xw = torch.ones(1, **f32)
-            self.inv_gx = torch.ones(1, **f32)
-            self.inv_gw = torch.ones(1, **f32)
             self.Xq = torch.empty((T, I), dtype=torch.float8_e4m3fn, device=dev)
             self.dYq = torch.empty((T, O), dtype=torch.float8_e5m2, device=dev)
+
+    def _amax(self, k):
+        return self.amax[k:k + 1] if self.fp8 else None
 
     # (0) first iteration only: beta is computed once and then frozen (Sec. 4.2)
     def init_beta(self):
@@ -60,13 +63,18 @@ class SsteLinear:
         self.beta_ready = True
         self.launches += 1
 
-    # (1) prune: w~ = beta * S_soft(W), compressed for the sparse products, dense for grad_X
+    # (1) prune: w~ = beta * S_soft(W), compressed for the sparse products (and for grad_X)
     def prune(self):
         assert self.beta_ready, "call init_beta() in the first iteration"
         c = self.ctx
         if self.track_flips:
             self.meta, self.meta_prev = self.meta_prev, self.meta     # last iteration's image becomes "previous"
-        self._project()
+        if self.fp8:
+            # the scale of w~ needs amax(w~) first: one read-only pass over W, then the cast to E4M3
+            c.project_amax(self.W, self.beta, self.amax[1:2])
+            self.launches += 1
+        c.project_compress(self.W, self.beta, self.vals, self.meta, self.w_dense, w_amax_dev=self._amax(1))
+        self.launches += 1
         if self.track_flips:
             if self._have_prev:
                 c.flip_count(self.meta_prev, self.meta, self.O, self.I, self.flips)
@@ -77,32 +85,19 @@ class SsteLinear:
         """r_k of the last prune (synchronises); 0 before the second prune."""
         return float(self.flips.item()) / (self.O * self.I)
 
-    def _project(self):
-        c = self.ctx
-        if not self.fp8:
-            c.project_compress(self.W, self.beta, self.vals, self.meta, self.w_dense)
-            self.launches += 1
-            return
-        # FP8: the scale of w~ needs amax(w~) first (one read-only pass over W), then the cast to E4M3
-        c.project_amax(self.W, self.beta, self.amax[1:2])
-        c.fp8_scale(self.amax[1:2], B.E4M3, self.scale[1:2], self.inv[1:2])
-        c.project_compress(self.W, self.beta, self.vals, self.meta, self.w_dense, wscale_dev=self.scale[1:2])
-        self.launches += 3
-
     # (2a) forward with the sparse weight
-    def forward(self, X):
+    def forward(self, X, y_amax_out=None):
         c = self.ctx
         if not self.fp8:
             self.X = X
-            c.linear_fwd(X, self.vals, self.meta, self.Y)
+            c.linear_fwd(X, self.vals, self.meta, self.Y, y_amax_out_dev=y_amax_out)
             self.launches += 1
             return self.Y
         c.amax(X, self.amax[0:1])
-        c.fp8_scale(self.amax[0:1], B.E4M3, self.scale[0:1], self.inv[0:1])
-        c.quantize_fp8(X, self.scale[0:1], self.Xq)
-        c.scalar_mul(self.inv[0:1], self.inv[1:2], self.inv_xw)
-        c.linear_fwd(self.Xq, self.vals, self.meta, self.Y, out_scale_dev=self.inv_xw)
-        self.launches += 5
+        c.quantize_fp8(X, self.amax[0:1], self.Xq)
+        c.linear_fwd(self.Xq, self.vals, self.meta, self.Y, x_amax_dev=self.amax[0:1], w_amax_dev=self.amax[1:2],
+                     y_amax_out_dev=y_amax_out)
+        self.launches += 3
         return self.Y
 
     # (2b) backward: MVUE on the output gradient for grad_W, dense product for grad_X
@@ -123,10 +118,12 @@ class SsteLinear:
         c = self.ctx
         if not hasattr(self, "wt_vals"):
             self.wt_vals, self.wt_meta = c.alloc_compressed(self.I, self.O, B.BF16)
+            self.wt_dense = torch.empty((self.O, self.I), dtype=torch.bfloat16, device=self.W.device)
         tid = self.tensor_id + (1 << 16) if tensor_id_w is None else tensor_id_w     # a stream of its own
-        c.mvue_sparsify(self.w_dense, self.seed, tid, step, self.wt_vals, self.wt_meta)
+        c.decompress(self.vals, self.meta, self.wt_dense)
+        c.mvue_sparsify(self.wt_dense, self.seed, tid, step, self.wt_vals, self.wt_meta)
         c.linear_fwd(dY, self.wt_vals, self.wt_meta, self.dX)
-        self.launches += 2
+        self.launches += 3
         return self.dX
 
     def grad_weight_and_input(self, dY, side_ctx: B.Context, side_stream: torch.cuda.Stream):
@@ -148,36 +145,78 @@ class SsteLinear:
     # (2b.1) MVUE(dY^T): 2:4 along tokens, compressed and transposed for the grad_W product
     def sparsify_grad(self, dY, step: int = 0, token_offset: int = 0):
         c = self.ctx
-        if not self.fp8:
-            c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta, token_offset=token_offset)
+        if self.fp8:
+            c.amax(dY, self.amax[2:3])
             self.launches += 1
-            return
-        c.amax(dY, self.amax[2:3])
-        c.fp8_scale(self.amax[2:3], B.E5M2, self.scale[2:3], self.inv[2:3])
-        c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta, dense_q_out=self.dYq,
-                        gscale_dev=self.scale[2:3], token_offset=token_offset)
-        self.launches += 3
+        c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta,
+                        dense_q_out=self.dYq if self.fp8 else None, g_amax_dev=self._amax(2),
+                        token_offset=token_offset, counter_cols=self.counter_cols)
+        self.launches += 1
 
     # (2b.2) grad_W = MVUE(dY^T) X, sparse
     def grad_weight(self):
-        c = self.ctx
-        if not self.fp8:
-            c.linear_bwd_weight(self.gvals, self.gmeta, self.X, self.dW)
-            self.launches += 1
-            return self.dW
-        c.scalar_mul(self.inv[2:3], self.inv[0:1], self.inv_gx)
-        c.linear_bwd_weight(self.gvals, self.gmeta, self.Xq, self.dW, out_scale_dev=self.inv_gx)
-        self.launches += 2
+        self.ctx.linear_bwd_weight(self.gvals, self.gmeta, self.Xq if self.fp8 else self.X, self.dW,
+                                   g_amax_dev=self._amax(2), x_amax_dev=self._amax(0))
+        self.launches += 1
         return self.dW
 
-    # (2b.3) grad_X = dY w~, dense
-    def grad_input(self, dY):
-        c = self.ctx
-        if not self.fp8:
-            c.linear_bwd_input(dY, self.w_dense, self.dX)
-            self.launches += 1
-            return self.dX
-        c.scalar_mul(self.inv[2:3], self.inv[1:2], self.inv_gw)
-        c.linear_bwd_input(self.dYq, self.w_dense, self.dX, out_scale_dev=self.inv_gw)
-        self.launches += 2
+    # (2b.3) grad_X = dY w~, dense; w~ from the compressed operand unless a dense copy is kept
+    def grad_input(self, dY, dx_amax_out=None):
+        g = self.dYq if self.fp8 else dY
+        if self.w_dense is not None:
+            self.ctx.linear_bwd_input(g, self.w_dense, self.dX, g_amax_dev=self._amax(2), w_amax_dev=self._amax(1),
+                                      dx_amax_out_dev=dx_amax_out)
+        else:
+            self.ctx.linear_bwd_input(g, None, self.dX, g_amax_dev=self._amax(2), w_amax_dev=self._amax(1),
+                                      vals=self.vals, meta=self.meta, dx_amax_out_dev=dx_amax_out)
+        self.launches += 1
         return self.dX
+
+
+class SsteLinearPadded:
+    """An S-STE linear of ANY shape (W[O, I], T tokens), run on zero-padded copies.
+
+    The library's kernels want multiples of 128.  Zero groups are fixed points of the projection (Eq. 4) and of
+    the MVUE rule and add nothing to beta, to an amax or to a product, so padding W, X and dY with zeros and
+    cropping Y, dX and dW gives the unpadded results; the MVUE counter runs over the unpadded column count.
+    The pad and crop passes are library kernels too (sste_pad_2d / sste_crop_2d).
+    """
+
+    def __init__(self, ctx: B.Context, O: int, I: int, T: int, **kw):
+        self.ctx, self.O, self.I, self.T = ctx, O, I, T
+        self.Op, self.Ip, self.Tp = B.padded_dim(O), B.padded_dim(I), B.padded_dim(T)
+        dev = f"cuda:{ctx.device}"
+        bf = dict(dtype=torch.bfloat16, device=dev)
+        self.Wp = torch.empty((self.Op, self.Ip), **bf)
+        self.Xp = torch.empty((self.Tp, self.Ip), **bf)
+        self.dYp = torch.empty((self.Tp, self.Op), **bf)
+        self.inner = SsteLinear(ctx, self.Wp, self.Tp, counter_cols=O, **kw)
+        self.Y = torch.empty((T, O), **bf)
+        self.dX = torch.empty((T, I), **bf)
+        self.dW = torch.empty((O, I), **bf)
+
+    @property
+    def beta(self):
+        return self.inner.beta
+
+    def set_weight(self, W):
+        self.ctx.pad_2d(W, self.Wp)
+
+    def init_beta(self):
+        self.inner.init_beta()
+
+    def prune(self):
+        self.inner.prune()
+
+    def forward(self, X):
+        self.ctx.pad_2d(X, self.Xp)
+        self.inner.forward(self.Xp)
+        self.ctx.crop_2d(self.inner.Y, self.Y)
+        return self.Y
+
+    def backward(self, dY, step: int = 0):
+        self.ctx.pad_2d(dY, self.dYp)
+        self.inner.backward(self.dYp, step=step)
+        self.ctx.crop_2d(self.inner.dX, self.dX)
+        self.ctx.crop_2d(self.inner.dW, self.dW)
+        return self.dX, self.dW

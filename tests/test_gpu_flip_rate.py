@@ -34,11 +34,11 @@ def test_flip_count_matches_the_definition(ctx, O, I, sigma, fp8):
     W1 = _perturbed(W0, sigma, 3) if sigma > 0 else W0.copy()
     dt = B.E4M3 if fp8 else B.BF16
     beta = torch.full((1,), 1.3, dtype=torch.float32, device=DEV)
-    one = torch.ones(1, dtype=torch.float32, device=DEV)
+    unit = torch.full((1,), 448.0, dtype=torch.float32, device=DEV)       # amax 448: E4M3 scale 1
     metas = []
     for W in (W0, W1):
         vals, meta = ctx.alloc_compressed(O, I, dt)
-        ctx.project_compress(dbf16(W), beta, vals, meta, None, wscale_dev=one if fp8 else None)
+        ctx.project_compress(dbf16(W), beta, vals, meta, None, w_amax_dev=unit if fp8 else None)
         metas.append(meta)
     count = torch.full((1,), -1, dtype=torch.int64, device=DEV)
     for _ in range(2):                                        # the call zeroes its own counter

@@ -45,15 +45,15 @@ def test_amax_scale_quantize(ctx):
         assert scale.item() == float(s_ref)
         assert inv.item() == float(np.float32(1.0) / s_ref)
         q = torch.empty(X.shape, dtype=tdt, device=DEV)
-        ctx.quantize_fp8(Xd, scale, q)
+        ctx.quantize_fp8(Xd, amax, q)                # the kernel forms the scale from the amax itself
         assert np.array_equal(bits8(q), orc.quantize(X, s_ref, dt))
     zero = dbf16(np.zeros((128, 128), np.uint16))
     ctx.amax(zero, amax)
     ctx.fp8_scale(amax, B.E4M3, scale, inv)
     assert (amax.item(), scale.item(), inv.item()) == (0.0, 1.0, 1.0)
-    a, b, out = _f32(0.3), _f32(7.0), _f32(0)
-    ctx.scalar_mul(a, b, out)
-    assert out.item() == float(np.float32(0.3) * np.float32(7.0))
+    q = torch.empty((128, 128), dtype=torch.float8_e4m3fn, device=DEV)
+    ctx.quantize_fp8(zero, amax, q)                  # amax = 0: scale 1, all codes +0
+    assert not bits8(q).any()
 
 
 @pytest.mark.parametrize("O,I", [(256, 256), (384, 640)])
@@ -63,17 +63,22 @@ def test_project_compress_e4m3(ctx, O, I):
     W[::5, ::3] = 0.0
     W[2] = 0.125
     W = synth.to_bf16_bits(W)
-    beta32, wscale = np.float32(1.4375), np.float32(5731.25)
+    beta32, w_amax = np.float32(1.4375), np.float32(0.078125)
+    wscale = orc.fp8_scale(w_amax, orc.E4M3)                       # the scale the kernel forms from the amax
     vals, meta = ctx.alloc_compressed(O, I, B.E4M3)
     dense = torch.empty((O, I), dtype=torch.float8_e4m3fn, device=DEV)
-    ctx.project_compress(dbf16(W), _f32(beta32), vals, meta, dense, wscale_dev=_f32(wscale))
+    ctx.project_compress(dbf16(W), _f32(beta32), vals, meta, dense, w_amax_dev=_f32(w_amax))
     ov, om, od = orc.project_compress(W, beta32, odt=orc.E4M3, wscale=wscale)
     assert np.array_equal(bits8(vals), ov)
     assert np.array_equal(canonical_meta(ctx, meta, O, I, B.E4M3), om)
     assert np.array_equal(bits8(dense), od)
-    # saturation: a huge scale clamps to +-448 instead of producing NaN codes
-    ctx.project_compress(dbf16(W), _f32(beta32), vals, meta, dense, wscale_dev=_f32(1e9))
-    assert np.array_equal(bits8(dense), orc.project_compress(W, beta32, odt=orc.E4M3, wscale=np.float32(1e9))[2])
+    dec = torch.empty_like(dense)
+    ctx.decompress(vals, meta, dec)
+    assert np.array_equal(bits8(dec), od)
+    # saturation: a far too small amax (a huge scale) clamps to +-448 instead of producing NaN codes
+    tiny = np.float32(448e-9)
+    ctx.project_compress(dbf16(W), _f32(beta32), vals, meta, dense, w_amax_dev=_f32(tiny))
+    assert np.array_equal(bits8(dense), orc.project_compress(W, beta32, odt=orc.E4M3, wscale=orc.fp8_scale(tiny, orc.E4M3))[2])
     assert not (bits8(dense) & 0x7F == 0x7F).any()
 
 
@@ -86,7 +91,7 @@ def test_mvue_e5m2(ctx, T, O):
     gscale = orc.fp8_scale(orc.amax(dY), orc.E5M2)
     gvals, gmeta = ctx.alloc_compressed(O, T, B.E5M2)
     dq = torch.empty((T, O), dtype=torch.float8_e5m2, device=DEV)
-    ctx.mvue_sparsify(dbf16(dY), 99, 4, 2, gvals, gmeta, dense_q_out=dq, gscale_dev=_f32(gscale))
+    ctx.mvue_sparsify(dbf16(dY), 99, 4, 2, gvals, gmeta, dense_q_out=dq, g_amax_dev=_f32(orc.amax(dY)))
     ogv, ogm, odq, _ = orc.mvue(dY, 99, 4, 2, odt=orc.E5M2, gscale=gscale, want_dense_q=True)
     assert np.array_equal(bits8(gvals), ogv)
     assert np.array_equal(canonical_meta(ctx, gmeta, O, T, B.E5M2), ogm)
@@ -97,7 +102,7 @@ def test_mvue_e5m2(ctx, T, O):
     assert np.array_equal(canonical_meta(ctx, m16, O, T, B.BF16), ogm)
 
 
-@pytest.mark.parametrize("tile_width", [0, 128, 192, 256])
+@pytest.mark.parametrize("tile_width", [0, 128, 192, 224, 256])
 @pytest.mark.parametrize("O,I,T", [(256, 256, 512), (384, 640, 1152), (128, 384, 128)])
 def test_fp8_products(ctx, O, I, T, tile_width):
     """Each product against the fp64 product of the decoded FP8 operands, times 1/(scale_a * scale_b)."""
@@ -107,17 +112,18 @@ def test_fp8_products(ctx, O, I, T, tile_width):
     dY = synth.gaussian_bf16(O + 13, (T, O), 1e-2)
     beta32 = np.float32(orc.beta(W)[0])
     _, _, wt16 = orc.project_compress(W, beta32)
+    aw, ax, ag = _f32(orc.amax(wt16)), _f32(orc.amax(X)), _f32(orc.amax(dY))
     sw = orc.fp8_scale(orc.amax(wt16), orc.E4M3)
     sx = orc.fp8_scale(orc.amax(X), orc.E4M3)
     sg = orc.fp8_scale(orc.amax(dY), orc.E5M2)
     vals, meta = ctx.alloc_compressed(O, I, B.E4M3)
     dense = torch.empty((O, I), dtype=torch.float8_e4m3fn, device=DEV)
-    ctx.project_compress(dbf16(W), _f32(beta32), vals, meta, dense, wscale_dev=_f32(sw))
+    ctx.project_compress(dbf16(W), _f32(beta32), vals, meta, dense, w_amax_dev=aw)
     Xq = torch.empty((T, I), dtype=torch.float8_e4m3fn, device=DEV)
-    ctx.quantize_fp8(dbf16(X), _f32(sx), Xq)
+    ctx.quantize_fp8(dbf16(X), ax, Xq)
     gvals, gmeta = ctx.alloc_compressed(O, T, B.E5M2)
     dYq = torch.empty((T, O), dtype=torch.float8_e5m2, device=DEV)
-    ctx.mvue_sparsify(dbf16(dY), 5, 0, 0, gvals, gmeta, dense_q_out=dYq, gscale_dev=_f32(sg))
+    ctx.mvue_sparsify(dbf16(dY), 5, 0, 0, gvals, gmeta, dense_q_out=dYq, g_amax_dev=ag)
     ctx.debug_force_tile_width(tile_width)
     inv_xw = np.float32(np.float32(1) / sx) * np.float32(np.float32(1) / sw)
     inv_gx = np.float32(np.float32(1) / sg) * np.float32(np.float32(1) / sx)
@@ -126,10 +132,15 @@ def test_fp8_products(ctx, O, I, T, tile_width):
         Y = torch.empty((T, O), dtype=odt, device=DEV)
         dW = torch.empty((O, I), dtype=odt, device=DEV)
         dX = torch.empty((T, I), dtype=odt, device=DEV)
-        ctx.linear_fwd(Xq, vals, meta, Y, out_scale_dev=_f32(inv_xw))
-        ctx.linear_bwd_weight(gvals, gmeta, Xq, dW, out_scale_dev=_f32(inv_gx))
-        ctx.linear_bwd_input(dYq, dense, dX, out_scale_dev=_f32(inv_gw))
+        ya = torch.full((1,), 1e9, device=DEV)
+        ctx.linear_fwd(Xq, vals, meta, Y, x_amax_dev=ax, w_amax_dev=aw, y_amax_out_dev=ya)
+        ctx.linear_bwd_weight(gvals, gmeta, Xq, dW, g_amax_dev=ag, x_amax_dev=ax)
+        ctx.linear_bwd_input(dYq, dense, dX, g_amax_dev=ag, w_amax_dev=aw)
+        dXc = torch.empty_like(dX)                   # the same product from the compressed E4M3 weight
+        ctx.linear_bwd_input(dYq, None, dXc, g_amax_dev=ag, w_amax_dev=aw, vals=vals, meta=meta)
         torch.cuda.synchronize()
+        assert torch.equal(dXc.view(torch.uint8), dX.view(torch.uint8))
+        assert ya.item() == Y.float().abs().max().item()
         Y_ref = orc.linear_fwd(bits8(Xq), orc.E4M3, bits8(vals), canonical_meta(ctx, meta, O, I, B.E4M3), orc.E4M3,
                                inv_scale=float(inv_xw))
         dW_ref = orc.linear_bwd_weight(bits8(gvals), canonical_meta(ctx, gmeta, O, T, B.E5M2), orc.E5M2, bits8(Xq),
@@ -150,7 +161,7 @@ def test_fp8_layer_end_to_end(ctx):
     from paper_2409_09099_b200.layer import SsteLinear
     O, I, T = 256, 384, 512
     W, X, dY = synth.gaussian_bf16(71, (O, I), 0.02), synth.gaussian_bf16(72, (T, I), 1.0), synth.gaussian_bf16(73, (T, O), 1e-2)
-    lin = SsteLinear(ctx, dbf16(W), T, tensor_id=3, seed=11, fp8=True)
+    lin = SsteLinear(ctx, dbf16(W), T, tensor_id=3, seed=11, fp8=True, dense_copy=True)
     lin.init_beta()
     lin.prune()
     Y = lin.forward(dbf16(X))
@@ -160,7 +171,7 @@ def test_fp8_layer_end_to_end(ctx):
     _, _, wt16 = orc.project_compress(W, beta32)
     sw, sx, sg = (orc.fp8_scale(orc.amax(wt16), orc.E4M3), orc.fp8_scale(orc.amax(X), orc.E4M3),
                   orc.fp8_scale(orc.amax(dY), orc.E5M2))
-    assert lin.scale.cpu().numpy().tolist() == [float(sx), float(sw), float(sg)]
+    assert lin.amax.cpu().numpy().tolist() == [orc.amax(X), orc.amax(wt16), orc.amax(dY)]
     ov, om, od = orc.project_compress(W, beta32, odt=orc.E4M3, wscale=sw)
     assert np.array_equal(bits8(lin.vals), ov) and np.array_equal(bits8(lin.w_dense), od)
     Xq = orc.quantize(X, sx, orc.E4M3)

@@ -118,7 +118,7 @@ def test_mvue_sparsify(ctx, O, I, T):
         ctx.mvue_sparsify(dbf16(dY), seed, tid, step, gvals, gmeta, token_offset=2)
 
 
-@pytest.fixture(params=[0, 128, 192, 256])
+@pytest.fixture(params=[0, 128, 192, 224, 256])
 def tile_width(request, ctx):
     """Every tile-width variant of the product kernels (0 = the library's own choice)."""
     ctx.debug_force_tile_width(request.param)
@@ -161,11 +161,24 @@ def test_three_products(ctx, O, I, T, out_dtype, tile_width):
         g = got.float().cpu().numpy().astype(np.float64)
         bound = 2.0 ** -7 * np.abs(ref) + 1e-4 * np.abs(ref).max()
         assert (np.abs(g - ref) <= bound).all()
-    # output scale factor
-    sc = torch.tensor([0.25], dtype=torch.float32, device=DEV)
+    # grad_X from the COMPRESSED weight (expanded inside the product) is the same product bit for bit, and the
+    # library's own decompression of the operand is the dense copy the projection wrote
+    dX2 = torch.full_like(dX, 7.0)
+    ctx.linear_bwd_input(dYd, None, dX2, vals=vals, meta=meta)
+    assert torch.equal(dX2.view(torch.int32 if out_dtype == torch.float32 else torch.int16),
+                       dX.view(torch.int32 if out_dtype == torch.float32 else torch.int16))
+    dec = torch.empty_like(dense)
+    ctx.decompress(vals, meta, dec)
+    assert torch.equal(dec.view(torch.int16), dense.view(torch.int16))
+    # optional amax outputs: max |Y|, max |grad_X| of the stored tensors (stale content must not matter)
+    ya, xa = torch.full((1,), 1e9, device=DEV), torch.full((1,), 1e9, device=DEV)
     Y2 = torch.empty_like(Y)
-    ctx.linear_fwd(Xd, vals, meta, Y2, out_scale_dev=sc)
-    assert torch.equal(Y2.float(), Y.float() * 0.25)
+    ctx.linear_fwd(Xd, vals, meta, Y2, y_amax_out_dev=ya)
+    ctx.linear_bwd_input(dYd, None, dX2, vals=vals, meta=meta, dx_amax_out_dev=xa)
+    assert torch.equal(Y2, Y)
+    assert ya.item() == Y.float().abs().max().item() and xa.item() == dX.float().abs().max().item()
+    if out_dtype == torch.bfloat16:
+        assert ya.item() == orc.amax(bits16(Y)) and xa.item() == orc.amax(bits16(dX))
 
 
 @pytest.mark.parametrize("splits", [1, 2, 3, 4])
@@ -193,7 +206,11 @@ def test_split_k_products(ctx, O, I, T, splits):
             ctx.linear_fwd(Xd, vals, meta, Y)
             ctx.linear_bwd_weight(gvals, gmeta, Xd, dW)
             ctx.linear_bwd_input(dYd, dense, dX)
+            dXc, xa = torch.empty_like(dX), torch.zeros(1, device=DEV)
+            ctx.linear_bwd_input(dYd, None, dXc, vals=vals, meta=meta, dx_amax_out_dev=xa)   # compressed weight, amax out
             torch.cuda.synchronize()
+            assert torch.equal(dXc.view(torch.int16), dX.view(torch.int16))
+            assert xa.item() == dX.float().abs().max().item()
             outs.append((Y, dW, dX))
     finally:
         ctx.debug_force_splits(0)

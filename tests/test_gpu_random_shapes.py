@@ -43,7 +43,9 @@ def test_layer_on_random_shape(ctx, O, I, T, fp8):
     X = synth.gaussian_bf16(I + 2, (T, I), 1.0)
     # groups of the gradient run along tokens: adversarial structure on the transposed view
     dY = np.ascontiguousarray(_adversarial(np.ascontiguousarray(synth.gaussian_bf16(T + 3, (T, O), 1e-2).T), rng).T)
-    lin = SsteLinear(ctx, dbf16(W), T, tensor_id=5, seed=77, fp8=fp8)
+    # half of the shapes keep a dense copy of w~ for grad_X, the others expand the compressed operand in the product
+    lin = SsteLinear(ctx, dbf16(W), T, tensor_id=5, seed=77, fp8=fp8, dense_copy=bool((O // 128) & 1))
+    dec = torch.empty((O, I), dtype=lin.vals.dtype, device=DEV)
     lin.init_beta(); lin.prune(); lin.forward(dbf16(X)); lin.backward(dbf16(dY), step=11)
     torch.cuda.synchronize()
     beta32 = np.float32(lin.beta.item())
@@ -51,7 +53,9 @@ def test_layer_on_random_shape(ctx, O, I, T, fp8):
     if not fp8:
         ov, om, od = orc.project_compress(W, beta32)
         ogv, ogm, _, _ = orc.mvue(dY, 77, 5, 11)
-        assert np.array_equal(bits16(lin.vals), ov) and np.array_equal(bits16(lin.w_dense), od)
+        ctx.decompress(lin.vals, lin.meta, dec)
+        assert np.array_equal(bits16(lin.vals), ov) and np.array_equal(bits16(dec), od)
+        assert lin.w_dense is None or np.array_equal(bits16(lin.w_dense), od)
         assert np.array_equal(canonical_meta(ctx, lin.meta, O, I, B.BF16), om)
         assert np.array_equal(bits16(lin.gvals), ogv)
         assert np.array_equal(canonical_meta(ctx, lin.gmeta, O, T, B.BF16), ogm)
@@ -65,7 +69,9 @@ def test_layer_on_random_shape(ctx, O, I, T, fp8):
         ov, om, od = orc.project_compress(W, beta32, odt=orc.E4M3, wscale=sw)
         Xq = orc.quantize(X, sx, orc.E4M3)
         ogv, ogm, odq, _ = orc.mvue(dY, 77, 5, 11, odt=orc.E5M2, gscale=sg, want_dense_q=True)
-        assert np.array_equal(bits8(lin.vals), ov) and np.array_equal(bits8(lin.w_dense), od)
+        ctx.decompress(lin.vals, lin.meta, dec)
+        assert np.array_equal(bits8(lin.vals), ov) and np.array_equal(bits8(dec), od)
+        assert lin.w_dense is None or np.array_equal(bits8(lin.w_dense), od)
         assert np.array_equal(canonical_meta(ctx, lin.meta, O, I, B.E4M3), om)
         assert np.array_equal(bits8(lin.gvals), ogv) and np.array_equal(bits8(lin.dYq), odq)
         assert np.array_equal(canonical_meta(ctx, lin.gmeta, O, T, B.E5M2), ogm)

@@ -37,14 +37,15 @@ def test_projection_variants(ctx, O, I, hard, gamma, fp8):
     from paper_2409_09099_b200 import binding as B
     W = _weights(O, I, O + I)
     beta32 = np.float32(1.0 if hard else 1.4837)
-    ws = np.float32(91.25)
+    w_amax = np.float32(4.90625)                       # the kernel forms the scale 448 / amax itself
+    ws = orc.fp8_scale(w_amax, orc.E4M3)
     dt = B.E4M3 if fp8 else B.BF16
     odt = orc.E4M3 if fp8 else orc.BF16
     beta = torch.full((1,), float(beta32), dtype=torch.float32, device=DEV)
-    wsd = torch.full((1,), float(ws), dtype=torch.float32, device=DEV)
+    wsd = torch.full((1,), float(w_amax), dtype=torch.float32, device=DEV)
     vals, meta = ctx.alloc_compressed(O, I, dt)
     dense = torch.empty((O, I), dtype=B._TORCH_DT[dt], device=DEV)
-    ctx.project_compress_variant(dbf16(W), beta, vals, meta, dense, wscale_dev=wsd if fp8 else None, hard=hard,
+    ctx.project_compress_variant(dbf16(W), beta, vals, meta, dense, w_amax_dev=wsd if fp8 else None, hard=hard,
                                  gamma=gamma)
     ov, om, od = orc.project_compress_variant(W, beta32, gamma=gamma, hard=hard, odt=odt, wscale=ws)
     bits = bits8 if fp8 else bits16
@@ -90,7 +91,8 @@ def test_srste_decay(ctx, fp8):
     dt = B.E4M3 if fp8 else B.BF16
     one = torch.ones(1, dtype=torch.float32, device=DEV)
     vals, meta = ctx.alloc_compressed(O, I, dt)
-    ctx.project_compress(dbf16(W), one, vals, meta, None, wscale_dev=one if fp8 else None)
+    unit = torch.full((1,), 448.0, dtype=torch.float32, device=DEV)       # amax 448: E4M3 scale 1
+    ctx.project_compress(dbf16(W), one, vals, meta, None, w_amax_dev=unit if fp8 else None)
     g = dbf16(dW)
     ctx.srste_decay(dbf16(W), meta, dt, lam, g)
     assert np.array_equal(bits16(g), orc.srste_decay(dW, W, lam))
