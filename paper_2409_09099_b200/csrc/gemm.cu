@@ -749,32 +749,46 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             lut[t] = sel;
         }
         asm volatile("bar.sync 2, 128;" ::: "memory");
-        const int n_half_vals = p.N / 2;                   // compressed values per row of B
-        const int n_atoms = p.N / 128;
-        int e_unit = pair, e_kb = 0, e_kend = 0, e_n0 = 0;
+        // A thread's units of a stage: the same 32-byte column segment `seg` of rows r0 + j * ROWS_STEP.
+        constexpr int ROWS_STEP = 128 / SEGS;
+        constexpr int EPU = 32 / ELT;                      // dense elements per unit
+        const int seg = t % SEGS, r0 = t / SEGS;
+        const size_t row_bytes = static_cast<size_t>(p.N / 2) * ELT;     // one row of compressed values
+        const size_t atom_row_bytes = static_cast<size_t>(p.N / 128) * 2048;
+        uint32_t moff[UNITS];                              // metadata byte of unit j inside its (half) atom
+#pragma unroll
+        for (int j = 0; j < UNITS; ++j) {
+            const uint32_t m = static_cast<uint32_t>(r0 + j * ROWS_STEP), k = static_cast<uint32_t>(seg * EPU);
+            moff[j] = F8 ? sste_meta_atom_byte8(m, k) : sste_meta_atom_byte16(m, k);
+        }
+        // loader cursor: (unit, stage) of the next loads
+        int e_unit = pair, e_kb = 0, e_kend = 0;
+        const uint8_t *e_vals = nullptr, *e_meta = nullptr;
+        bool e_cols = false;
         auto e_setup = [&]() {
             if (e_unit >= num_units) return;
             const Unit u = decode(e_unit);
-            e_n0 = (u.tile / m_tiles) * BN + static_cast<int>(rank) * (BN / 2);
+            const int n0 = (u.tile / m_tiles) * BN + static_cast<int>(rank) * (BN / 2);
+            e_cols = n0 < p.N;
+            e_vals = p.b_vals + (static_cast<size_t>(n0 / 2) + seg * (EPU / 2)) * ELT + r0 * row_bytes;
+            e_meta = meta + static_cast<size_t>(n0 >> 7) * 2048;
             e_kb = u.split * u.k_blocks;
             e_kend = e_kb + u.k_blocks;
         };
         auto e_issue = [&](uint4 (&v)[UNITS], uint32_t (&m)[UNITS]) -> bool {
             if (e_unit >= num_units) return false;
+            const uint32_t krow0 = static_cast<uint32_t>(e_kb) * BK;             // first K row of the stage
+            const uint8_t *vp = e_vals + krow0 * row_bytes;
+            const uint8_t *mp = e_meta + (krow0 >> 7) * atom_row_bytes + ((BK == 64 && (krow0 & 64u)) ? 1024u : 0u);
 #pragma unroll
             for (int j = 0; j < UNITS; ++j) {
-                const int un = j * 128 + t;
-                const uint32_t krow = static_cast<uint32_t>(e_kb * BK + un / SEGS);
-                const uint32_t ncol = static_cast<uint32_t>(e_n0 + (un % SEGS) * (32 / ELT));
-                if (ncol < static_cast<uint32_t>(p.N) && krow < static_cast<uint32_t>(p.K)) {
-                    v[j] = __ldg(reinterpret_cast<const uint4 *>(
-                        p.b_vals + (static_cast<size_t>(krow) * n_half_vals + ncol / 2) * ELT));
-                    const uint8_t *atom = meta + (static_cast<size_t>(krow >> 7) * n_atoms + (ncol >> 7)) * 2048;
-                    if (F8) m[j] = __ldg(reinterpret_cast<const uint32_t *>(atom + sste_meta_atom_byte8(krow & 127u, ncol & 127u)));
-                    else m[j] = __ldg(reinterpret_cast<const uint16_t *>(atom + sste_meta_atom_byte16(krow & 127u, ncol & 127u)));
+                if (e_cols) {
+                    v[j] = __ldg(reinterpret_cast<const uint4 *>(vp + static_cast<size_t>(j) * ROWS_STEP * row_bytes));
+                    if (F8) m[j] = __ldg(reinterpret_cast<const uint32_t *>(mp + moff[j]));
+                    else m[j] = __ldg(reinterpret_cast<const uint16_t *>(mp + moff[j]));
                 } else {
-                    v[j] = make_uint4(0, 0, 0, 0);
-                    m[j] = 0x44444444u;                    // any valid code: the values are zero
+                    v[j] = make_uint4(0, 0, 0, 0);         // columns beyond N: zeros (any valid code will do)
+                    m[j] = 0x44444444u;
                 }
             }
             if (++e_kb >= e_kend) {
@@ -784,38 +798,38 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             return true;
         };
         e_setup();
-        uint4 cv[UNITS], nv[UNITS];
-        uint32_t cm[UNITS], nm[UNITS];
-        bool have = e_issue(cv, cm);
+        // three stages of loads in flight in registers: a round trip to L2 is longer than two stages of MMAs
+        uint4 v0[UNITS], v1[UNITS], v2[UNITS];
+        uint32_t m0[UNITS], m1[UNITS], m2[UNITS];
+        bool h0 = e_issue(v0, m0), h1 = e_issue(v1, m1), h2 = e_issue(v2, m2);
         uint32_t it = 0;
-        while (have) {
-            const bool have_next = e_issue(nv, nm);
+        uint8_t *const ring = smem_raw + (smem_base - smem_u32(smem_raw));
+        while (h0) {
             const int s = it % NS;
             const uint32_t ph = (it / NS) & 1u;
             if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, p.status, abort_flag)) break;
-            uint8_t *b_dst = smem_raw + (smem_base - smem_u32(smem_raw)) + s * C::STAGE + C::A_STAGE;
+            uint8_t *b_dst = ring + s * C::STAGE + C::A_STAGE + (seg >> 2) * (BK * 128);
+            const int j0 = (seg & 3) * 2;
 #pragma unroll
             for (int j = 0; j < UNITS; ++j) {
-                const int un = j * 128 + t;
-                const int r = un / SEGS, seg = un % SEGS;
-                const uint32_t w[4] = {cv[j].x, cv[j].y, cv[j].z, cv[j].w};
+                const int r = r0 + j * ROWS_STEP;
+                const uint32_t w[4] = {v0[j].x, v0[j].y, v0[j].z, v0[j].w};
                 uint32_t o[8];
                 if (F8) {
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
                         const uint32_t pairw = (g & 1) ? (w[g >> 1] >> 16) : w[g >> 1];    // value bytes 0, 1
-                        o[g] = __byte_perm(pairw, 0, lut[(cm[j] >> (4 * g)) & 0xfu]);
+                        o[g] = __byte_perm(pairw, 0, lut[(m0[j] >> (4 * g)) & 0xfu]);
                     }
                 } else {
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
-                        const uint32_t sel = lut[(cm[j] >> (4 * g)) & 0xfu];
+                        const uint32_t sel = lut[(m0[j] >> (4 * g)) & 0xfu];
                         o[2 * g] = __byte_perm(w[g], 0, sel & 0xffffu);
                         o[2 * g + 1] = __byte_perm(w[g], 0, sel >> 16);
                     }
                 }
-                uint8_t *rowp = b_dst + (seg >> 2) * (BK * 128) + r * 128;
-                const int j0 = (seg & 3) * 2;
+                uint8_t *rowp = b_dst + r * 128;
                 *reinterpret_cast<uint4 *>(rowp + ((j0 ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
                 *reinterpret_cast<uint4 *>(rowp + (((j0 + 1) ^ (r & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
             }
@@ -823,8 +837,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(full_bar(s), 0));
 #pragma unroll
-            for (int j = 0; j < UNITS; ++j) { cv[j] = nv[j]; cm[j] = nm[j]; }
-            have = have_next;
+            for (int j = 0; j < UNITS; ++j) { v0[j] = v1[j]; m0[j] = m1[j]; v1[j] = v2[j]; m1[j] = m2[j]; }
+            h0 = h1;
+            h1 = h2;
+            h2 = e_issue(v2, m2);
             ++it;
         }
     }
@@ -1024,21 +1040,32 @@ SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int alig
     return SplitPlan{best, whole};
 }
 
-// Tile width, from timings on B200 over the GPT-2- and 7B-shaped layers: 256 columns is the fastest
-// almost everywhere (least L2 -> shared-memory traffic per flop); the forward gains from 192 columns
-// with a short reduction (K <= 1024), where the second accumulator buffer hides an epilogue that is as
-// long as the main loop, and when 256-wide tiles leave most of the last wave empty.
-int pick_bn(bool b_k_major, int M, int N, int K, int pairs)
+// Tile width of the forward (K-major B), from timings on B200 over the GPT-2- and 7B-shaped layers.
+// bf16: the time of a tile is close to  K * bn * k(bn) + f(bn)  microseconds with
+//   bn = 192: k = 1.93e-5, f = 0.4;   224: k = 1.83e-5, f = 0.5;   256: k = 1.52e-5, f = 1.7
+// (wider tiles stream less B per flop; the 256-wide tile has one accumulator, so its epilogue is exposed), and
+// the launch takes ceil(tiles / pairs) such tile times: the width with the smallest product wins, which is
+// mostly a matter of how the tile count quantises into waves.  FP8: 256 columns unless they quantise badly.
+int pick_bn(bool b_k_major, int elt, int M, int N, int K, int pairs)
 {
     if (!b_k_major) return 256;
-    if (K <= 1024) return 192;
-    // Longer reductions: 256 columns unless the tile count quantises badly (GPT-2 fc2 forward: 96 tiles on
-    // 74 CTA pairs are two waves; 129 tiles of 192 columns are two waves of 3/4 the work).  A 192-wide tile
-    // costs about 8 % more per flop (measured at many waves).
     const long m_tiles = (M + 2 * BM - 1) / (2 * BM);
-    const long waves256 = (m_tiles * ((N + 255) / 256) + pairs - 1) / pairs;
-    const long waves192 = (m_tiles * ((N + 191) / 192) + pairs - 1) / pairs;
-    return (waves192 * 192 * 108 < waves256 * 256 * 100) ? 192 : 256;
+    auto waves = [&](int bn) { return (m_tiles * ((N + bn - 1) / bn) + pairs - 1) / pairs; };
+    if (elt == 2) {
+        const int widths[3] = {224, 192, 256};
+        const double k[3] = {1.83e-5, 1.93e-5, 1.52e-5}, f[3] = {0.5, 0.4, 1.7};
+        int best = 0;
+        double best_cost = 0.0;
+        for (int i = 0; i < 3; ++i) {
+            const double cost = static_cast<double>(waves(widths[i])) * (static_cast<double>(K) * widths[i] * k[i] + f[i]);
+            if (i == 0 || cost < best_cost * 0.995) { best = i; best_cost = cost; }
+        }
+        return widths[best];
+    }
+    if (K <= 1024) return 192;
+    // Longer reductions: 256 columns unless the tile count quantises badly; a 192-wide tile costs about 8 %
+    // more per flop (measured at many waves).
+    return (waves(192) * 192 * 108 < waves(256) * 256 * 100) ? 192 : 256;
 }
 
 bool fmt_code(sste_dtype dt, int *elt, uint32_t *code)
@@ -1066,7 +1093,7 @@ sste_status launch_out(const sste_ctx *ctx, const void *A, const void *B, const 
     if (!(MN && ELT == 1)) cands[n++] = 128;   // MN-major B: each CTA needs whole 128-byte chunks of N
     if (!MN) cands[n++] = 192;
     if (!MN && SPARSE && OUT_T) cands[n++] = 224;
-    int bn = pick_bn(!MN, p.M, p.N, p.K, ctx->sm_count / 2);
+    int bn = pick_bn(!MN, ELT, p.M, p.N, p.K, ctx->sm_count / 2);
     for (int i = 0; i < n; ++i)
         if (cands[i] == g_force_bn) bn = g_force_bn;
     if constexpr (!MN && SPARSE && OUT_T) {

@@ -18,15 +18,16 @@ class SsteLinear:
     ``fp8=True`` selects the whole-process FP8 variant (Sec. 5.2): E4M3 forward
     operands, E5M2 output gradient, per-tensor scale = fp8_max / amax; the state of a
     quantised tensor is its amax (one device float), from which every consumer forms the
-    scale itself.  ``dense_copy=True`` also keeps w~ as a dense [O, I] tensor and feeds
-    grad_X from it; by default grad_X expands the compressed operand inside the product.
+    scale itself.  ``dense_copy=True`` (the default, the faster route on B200) also keeps w~ as a
+    dense [O, I] tensor and feeds grad_X from it; with ``dense_copy=False`` no dense w~ exists and
+    grad_X expands the compressed operand inside the product (same bits, less memory, slower).
     ``track_flips=True`` keeps the previous iteration's metadata and counts the mask entries
     that changed at every prune (flip rate, Sec. 3.1).
     """
 
     def __init__(self, ctx: B.Context, W: torch.Tensor, T: int, tensor_id: int = 0, seed: int = 0,
                  fp8: bool = False, out_dtype: torch.dtype = torch.bfloat16, track_flips: bool = False,
-                 dense_copy: bool = False, counter_cols: int = 0):
+                 dense_copy: bool = True, counter_cols: int = 0):
         assert W.dtype == torch.bfloat16 and W.is_cuda
         self.ctx, self.W, self.T, self.tensor_id, self.seed, self.fp8 = ctx, W, T, tensor_id, seed, fp8
         self.O, self.I = W.shape
@@ -44,6 +45,7 @@ class SsteLinear:
         self.dX = torch.empty((T, I), dtype=out_dtype, device=dev)
         self.dW = torch.empty((O, I), dtype=out_dtype, device=dev)
         self.launches = 0
+        self.mark = None       # optional callback(label), called before every C-ABI call (a benchmark records events)
         self.track_flips = track_flips
         if track_flips:
             self.meta_prev = torch.empty_like(self.meta)
@@ -56,6 +58,10 @@ class SsteLinear:
 
     def _amax(self, k):
         return self.amax[k:k + 1] if self.fp8 else None
+
+    def _m(self, label):
+        if self.mark is not None:
+            self.mark(label)
 
     # (0) first iteration only: beta is computed once and then frozen (Sec. 4.2)
     def init_beta(self):
@@ -71,12 +77,15 @@ class SsteLinear:
             self.meta, self.meta_prev = self.meta_prev, self.meta     # last iteration's image becomes "previous"
         if self.fp8:
             # the scale of w~ needs amax(w~) first: one read-only pass over W, then the cast to E4M3
+            self._m("project_amax")
             c.project_amax(self.W, self.beta, self.amax[1:2])
             self.launches += 1
+        self._m("project_compress")
         c.project_compress(self.W, self.beta, self.vals, self.meta, self.w_dense, w_amax_dev=self._amax(1))
         self.launches += 1
         if self.track_flips:
             if self._have_prev:
+                self._m("flip_count")
                 c.flip_count(self.meta_prev, self.meta, self.O, self.I, self.flips)
                 self.launches += 1
             self._have_prev = True
@@ -90,11 +99,15 @@ class SsteLinear:
         c = self.ctx
         if not self.fp8:
             self.X = X
+            self._m("linear_fwd")
             c.linear_fwd(X, self.vals, self.meta, self.Y, y_amax_out_dev=y_amax_out)
             self.launches += 1
             return self.Y
+        self._m("amax_x")
         c.amax(X, self.amax[0:1])
+        self._m("quantize_x")
         c.quantize_fp8(X, self.amax[0:1], self.Xq)
+        self._m("linear_fwd")
         c.linear_fwd(self.Xq, self.vals, self.meta, self.Y, x_amax_dev=self.amax[0:1], w_amax_dev=self.amax[1:2],
                      y_amax_out_dev=y_amax_out)
         self.launches += 3
@@ -146,8 +159,10 @@ class SsteLinear:
     def sparsify_grad(self, dY, step: int = 0, token_offset: int = 0):
         c = self.ctx
         if self.fp8:
+            self._m("amax_g")
             c.amax(dY, self.amax[2:3])
             self.launches += 1
+        self._m("mvue_sparsify")
         c.mvue_sparsify(dY, self.seed, self.tensor_id, step, self.gvals, self.gmeta,
                         dense_q_out=self.dYq if self.fp8 else None, g_amax_dev=self._amax(2),
                         token_offset=token_offset, counter_cols=self.counter_cols)
@@ -155,6 +170,7 @@ class SsteLinear:
 
     # (2b.2) grad_W = MVUE(dY^T) X, sparse
     def grad_weight(self):
+        self._m("linear_bwd_weight")
         self.ctx.linear_bwd_weight(self.gvals, self.gmeta, self.Xq if self.fp8 else self.X, self.dW,
                                    g_amax_dev=self._amax(2), x_amax_dev=self._amax(0))
         self.launches += 1
@@ -163,6 +179,7 @@ class SsteLinear:
     # (2b.3) grad_X = dY w~, dense; w~ from the compressed operand unless a dense copy is kept
     def grad_input(self, dY, dx_amax_out=None):
         g = self.dYq if self.fp8 else dY
+        self._m("linear_bwd_input")
         if self.w_dense is not None:
             self.ctx.linear_bwd_input(g, self.w_dense, self.dX, g_amax_dev=self._amax(2), w_amax_dev=self._amax(1),
                                       dx_amax_out_dev=dx_amax_out)

@@ -30,3 +30,32 @@ def test_reference_arm_prints_one_json_line():
 def test_reference_arm_other_ranks_print_nothing():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2")
     assert _run("--impl", "reference", "--gpus", "2", "--config", "1", "--steps", "1", "--warmup", "0", env=env) == []
+
+
+def test_reference_arm_with_gpus_flag_prints_one_line_from_one_process():
+    """`--gpus 2 --impl reference` outside torchrun: one process, one line, n_gpus echoed."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    lines = _run("--impl", "reference", "--gpus", "2", "--config", "1", "--steps", "1", "--warmup", "0",
+                 "--ref-tokens", "128", env=env)
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2
+
+
+def test_spawn_command_starts_one_rank_per_gpu(monkeypatch):
+    """`--gpus N` without a torchrun environment re-launches bench.py under torch.distributed.run with N ranks."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("bench_mod", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    seen = {}
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: seen.setdefault("cmd", cmd) and 0)
+    monkeypatch.setattr(bench.sys, "argv", ["bench.py", "--gpus", "4", "--steps", "3"])
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    try:
+        bench.main()
+    except SystemExit as e:
+        assert e.code == 0
+    cmd = seen["cmd"]
+    assert "torch.distributed.run" in cmd and "--nproc-per-node=4" in cmd and "127.0.0.1" in cmd
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "3"]

@@ -32,7 +32,7 @@ def ctx():
 
 
 def _run_layer(ctx, W, X, dY, tensor_id, seed, step, fp8):
-    """The layer as bench.py runs it: grad_X from the compressed weight, no dense copy of w~ on the path."""
+    """The layer as bench.py runs it (library defaults)."""
     from paper_2409_09099_b200.layer import SsteLinear
     lin = SsteLinear(ctx, dbf16(W), X.shape[0], tensor_id=tensor_id, seed=seed, fp8=fp8)
     lin.init_beta()
@@ -54,7 +54,7 @@ def test_config2_full(ctx, layer):
     beta_ref = orc.beta(W)[0]
     assert abs(lin.beta.item() - beta_ref) <= 1e-6 * beta_ref
     ov, om, od = orc.project_compress(W, np.float32(lin.beta.item()))
-    assert np.array_equal(bits16(lin.vals), ov)
+    assert np.array_equal(bits16(lin.vals), ov) and np.array_equal(bits16(lin.w_dense), od)
     assert np.array_equal(canonical_meta(ctx, lin.meta, O, I, B.BF16), om)
     ogv, ogm, _, _ = orc.mvue(dY, cfg["seed"], layer, 3)
     assert np.array_equal(bits16(lin.gvals), ogv)
@@ -98,7 +98,7 @@ def _bf16_layer_sampled(ctx, cfg_id, layer, rng_seed):
     beta_ref = orc.beta(W)[0]
     assert abs(lin.beta.item() - beta_ref) <= 1e-6 * beta_ref
     ov, om, od = orc.project_compress(W, np.float32(lin.beta.item()))
-    assert np.array_equal(bits16(lin.vals), ov)
+    assert np.array_equal(bits16(lin.vals), ov) and np.array_equal(bits16(lin.w_dense), od)
     assert np.array_equal(canonical_meta(ctx, lin.meta, O, I, B.BF16), om)
     ogv, ogm, _, _ = orc.mvue(dY, cfg["seed"], layer, 0)
     assert np.array_equal(bits16(lin.gvals), ogv)
@@ -137,7 +137,7 @@ def test_config5_fp8_every_layer_sampled(ctx, layer):
                   orc.fp8_scale(orc.amax(dY), orc.E5M2))
     assert lin.amax.cpu().numpy().tolist() == [orc.amax(X), orc.amax(wt16), orc.amax(dY)]
     ov, om, od = orc.project_compress(W, beta32, odt=orc.E4M3, wscale=sw)
-    assert np.array_equal(bits8(lin.vals), ov)
+    assert np.array_equal(bits8(lin.vals), ov) and np.array_equal(bits8(lin.w_dense), od)
     assert np.array_equal(canonical_meta(ctx, lin.meta, O, I, B.E4M3), om)
     Xq = orc.quantize(X, sx, orc.E4M3)
     assert np.array_equal(bits8(lin.Xq), Xq)
