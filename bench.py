@@ -613,6 +613,51 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_model(args):
+    """--config 4: training steps of the 12-layer GPT-2-124M-shaped decoder with every linear through libsste."""
+    import torch
+
+    from paper_2409_09099_b200 import binding as B
+    from paper_2409_09099_b200.model import SsteGpt2, synthetic_batch
+    torch.cuda.set_device(0)
+    sampler = ClockSampler(0)
+    sampler.start()
+    ctx = B.Context(0)
+    model = SsteGpt2(ctx)
+    tokens, targets = synthetic_batch(model, 4)
+    for _ in range(max(args.warmup, 3)):
+        model.train_step(tokens, targets)
+    torch.cuda.synchronize()
+    n0, t0 = B.launch_count(), time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        loss, _ = model.train_step(tokens, targets)
+    e1.record()
+    torch.cuda.synchronize()
+    t1, launches = time.time(), B.launch_count() - n0
+    ms = e0.elapsed_time(e1) / args.steps
+    inside, total = 0.0, 0.0
+    for _ in range(3):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        _, t_in = model.train_step(tokens, targets, time_libsste=True)
+        b.record()
+        torch.cuda.synchronize()
+        inside, total = inside + t_in, total + a.elapsed_time(b) * 1e-3
+    status = ctx.poll_device_status()
+    sampler.stop()
+    line = {"metric": METRIC, "value": model.flops_per_step() / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "BASELINE config 4: 12-layer GPT-2-124M-shaped decoder, 8 x 1024 uniform token ids, all 48 "
+                                   "linears through libsste; attention, layer norms, embeddings, loss and AdamW in torch",
+                       "note": "value counts the S-STE linears' 6*T*I*O flops over the WHOLE training step"},
+            "libsste_fraction_of_step": inside / total, "loss": float(loss), "gpu_launches": int(launches),
+            "clocks": sampler.window(t0, t1), "device_status": status}
+    print(json.dumps(line), flush=True)
+
+
 def spawn_ranks(args):
     """`--gpus N` outside a torchrun environment: start the N ranks (one per GPU) and let rank 0 print."""
     with socket.socket() as s:
@@ -641,6 +686,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.config == 4:
+        run_model(args)
     elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         spawn_ranks(args)
     else:
