@@ -330,6 +330,14 @@ sste_status sste_debug_force_tile_width(int bn);
  * falls back to the automatic choice. */
 sste_status sste_debug_force_splits(int splits);
 
+/* Test hook for the bounded waits.  While armed (on != 0), a dense sste_linear_bwd_input (Wt_dense given, bf16
+ * output) whose output is ONE tile (T <= 256, I <= 256) leaves the last K stage of its operand pipeline unloaded
+ * and limits every device-side wait to one millisecond instead of two seconds: the wait for that stage runs out,
+ * the kernel records SSTE_ERR_TIMEOUT in the status word, abandons the tile and returns (dX is not written).
+ * Nothing traps or spins, the context stays usable.  Any other product call returns SSTE_ERR_INVALID_ARG while
+ * the hook is armed.  Process-wide; disarm with 0. */
+sste_status sste_debug_inject_stall(int on);
+
 #ifdef __cplusplus
 }
 #endif

@@ -30,7 +30,7 @@ EXPORTS = [
     "sste_quantize_fp8", "sste_meta_to_canonical", "sste_debug_force_tile_width", "sste_debug_force_splits",
     "sste_workspace_bytes_recommended", "sste_beta_init_static", "sste_debug_launch_count", "sste_flip_count",
     "sste_project_compress_variant", "sste_beta_init_l1", "sste_srste_decay", "sste_project_amax",
-    "sste_decompress", "sste_padded_dim", "sste_pad_2d", "sste_crop_2d",
+    "sste_decompress", "sste_padded_dim", "sste_pad_2d", "sste_crop_2d", "sste_debug_inject_stall",
 ]
 
 
@@ -238,6 +238,9 @@ class Context:
 
     def debug_force_splits(self, splits: int):
         self._check(self.lib.sste_debug_force_splits(splits))
+
+    def debug_inject_stall(self, on: bool):
+        self._check(self.lib.sste_debug_inject_stall(1 if on else 0))
 
     def debug_force_tile_width(self, bn: int):
         self._check(self.lib.sste_debug_force_tile_width(bn))

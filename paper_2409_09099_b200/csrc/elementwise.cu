@@ -464,19 +464,24 @@ mvue_kernel(const uint4 *__restrict__ dY, int O, int T, uint32_t key0, uint32_t 
 __global__ void __launch_bounds__(EW_THREADS)
 amax_kernel(const uint4 *__restrict__ x, size_t n_chunks, float *__restrict__ amax_dev)
 {
-    uint32_t best = 0;   // magnitude bits of bf16 compare like unsigned integers
+    uint32_t best2 = 0;   // magnitude bits of bf16 compare like unsigned integers: running maximum in both halves
     sste_pdl_trigger();
     sste_pdl_wait();
-    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
-         c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
-        const uint4 v = __ldg(x + c);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    // four independent 16-byte loads per thread and iteration: a pure read needs the bytes in flight
+    const size_t stride = static_cast<size_t>(gridDim.x) * EW_THREADS;
+    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks; c += 4 * stride) {
+        uint4 v[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            best = max(best, w[i] & 0x7fffu);
-            best = max(best, (w[i] >> 16) & 0x7fffu);
+        for (int j = 0; j < 4; ++j) v[j] = (c + j * stride < n_chunks) ? __ldg(x + c + j * stride) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            best2 = __vmaxu2(best2, v[j].x & 0x7fff7fffu);
+            best2 = __vmaxu2(best2, v[j].y & 0x7fff7fffu);
+            best2 = __vmaxu2(best2, v[j].z & 0x7fff7fffu);
+            best2 = __vmaxu2(best2, v[j].w & 0x7fff7fffu);
         }
     }
+    uint32_t best = max(best2 & 0xffffu, best2 >> 16);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
     if ((threadIdx.x & 31) == 0 && best != 0)
@@ -493,14 +498,24 @@ project_amax_kernel(const uint4 *__restrict__ W, size_t n_chunks, const float *_
     sste_pdl_wait();
     const float beta = *beta_dev;
     float best = 0.0f;
-    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
-         c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
-        const uint4 v = __ldg(W + c);
-        const uint32_t raw[4] = {v.x, v.y, v.z, v.w};
+    const size_t stride = static_cast<size_t>(gridDim.x) * EW_THREADS;
+    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks; c += 4 * stride) {
+        uint4 v[4];
 #pragma unroll
-        for (int g = 0; g < 2; ++g) {
-            const SoftGroup s = soft_group<false, 0>(raw[2 * g], raw[2 * g + 1], beta, 1.0f, 0.0f);
-            best = fmaxf(best, fmaxf(fmaxf(fabsf(s.w[0]), fabsf(s.w[1])), fmaxf(fabsf(s.w[2]), fabsf(s.w[3]))));
+        for (int j = 0; j < 4; ++j) v[j] = (c + j * stride < n_chunks) ? __ldg(W + c + j * stride) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t raw[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                // the largest |w~| of a group belongs to its largest |w|: one product per group suffices
+                const uint32_t m01 = raw[2 * g] & 0x7fff7fffu, m23 = raw[2 * g + 1] & 0x7fff7fffu;
+                const uint32_t lo = __vminu2(m01, m23), hi = __vmaxu2(m01, m23);
+                const uint32_t t2 = __vminu2(__vmaxu2(lo, __byte_perm(lo, 0, 0x1032)), __vminu2(hi, __byte_perm(hi, 0, 0x1032)));
+                const uint32_t mx = __vmaxu2(hi, __byte_perm(hi, 0, 0x1032));
+                const float d = __fsub_rn(__uint_as_float(mx << 16), __uint_as_float(t2 << 16));
+                best = fmaxf(best, fabsf(__fmul_rn(d, beta)));
+            }
         }
     }
 #pragma unroll
@@ -528,20 +543,24 @@ quantize_kernel(const uint4 *__restrict__ x, size_t n_chunks, const float *__res
     sste_pdl_trigger();
     sste_pdl_wait();
     const float scale = sste_scale_from_amax(*amax_dev, E5M2 ? 57344.0f : 448.0f);
-    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks;
-         c += static_cast<size_t>(gridDim.x) * EW_THREADS) {
-        const uint4 v = __ldg(x + c);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        uint32_t b[8];
+    const size_t stride = static_cast<size_t>(gridDim.x) * EW_THREADS;
+    for (size_t c = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; c < n_chunks; c += 4 * stride) {
+        uint4 v[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float f = __fmul_rn(sste_bf16_bits_to_f32((i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xffffu)), scale);
-            b[i] = E5M2 ? sste_f32_to_e5m2(f) : sste_f32_to_e4m3(f);
+        for (int j = 0; j < 4; ++j) v[j] = (c + j * stride < n_chunks) ? __ldg(x + c + j * stride) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (c + j * stride >= n_chunks) break;
+            const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+            uint32_t h[4];           // two codes per word: packed conversion of (low half, high half)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = make_float2(__fmul_rn(__uint_as_float(w[i] << 16), scale),
+                                             __fmul_rn(__uint_as_float(w[i] & 0xffff0000u), scale));
+                h[i] = static_cast<uint32_t>(__nv_cvt_float2_to_fp8x2(f, __NV_SATFINITE, E5M2 ? __NV_E5M2 : __NV_E4M3));
+            }
+            q[c + j * stride] = make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
         }
-        uint2 d;
-        d.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
-        d.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
-        q[c] = d;
     }
 }
 

@@ -87,25 +87,30 @@ __device__ __forceinline__ unsigned long long global_ns()
 }
 // Bounded wait of ONE thread.  Returns false (after recording a timeout) instead of spinning forever.
 // The limit is wall time (nanoseconds of %globaltimer), so it does not depend on the SM clock.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned int *status, volatile int *abort_flag)
+struct WaitCtx {
+    unsigned int *status;              // the context's device status word
+    volatile int *abort_flag;          // this CTA's "a wait has expired" flag (shared memory)
+    unsigned long long limit_ns;       // WAIT_LIMIT_NS, or the short limit of the stall-injection test hook
+};
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx &wc)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long start = global_ns();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_ns() - start > WAIT_LIMIT_NS) {
-            atomicCAS(status, 0u, static_cast<unsigned int>(SSTE_ERR_TIMEOUT));
-            *abort_flag = 1;
+        if (*wc.abort_flag) return false;
+        if (global_ns() - start > wc.limit_ns) {
+            atomicCAS(wc.status, 0u, static_cast<unsigned int>(SSTE_ERR_TIMEOUT));
+            *wc.abort_flag = 1;
             return false;
         }
     }
 }
 // Bounded wait of a whole warp: lane 0 waits, the others park at the warp barrier.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, unsigned int *status, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitCtx &wc)
 {
     uint32_t ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, status, abort_flag) ? 1u : 0u;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, wc) ? 1u : 0u;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     return ok != 0;
 }
@@ -247,6 +252,8 @@ struct GemmParams {
     unsigned int *status;
     uint32_t afmt, bfmt;    // operand format codes of the instruction descriptor
     const uint8_t *b_vals;  // compressed-B kernels: the 2:4 values of B [K, N/2]; its metadata image is `meta`
+    unsigned long long wait_limit_ns;   // limit of every device-side wait
+    int skip_last_stage;    // stall-injection test hook: the producer leaves the last K stage of the launch unloaded
     int splits;             // split-K factor of the tiles from `split_from` on (1 = none)
     int split_from;         // first split tile: tiles below it are computed whole
     float *partials;        // split-K: fp32 partial tiles [tile][cta][split][128][BN], summed by splitk_reduce_kernel
@@ -330,6 +337,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_generic + 8u * (MISC + 1));
     uint8_t *staging_generic = smem_raw + (staging - smem_u32(smem_raw));
     static_assert(8 * (MISC + 2) + 64 <= 512, "barrier block (+ the expander's 16-entry selector table)");
+    const WaitCtx wc{p.status, abort_flag, p.wait_limit_ns};
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -393,7 +401,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 for (int kb = kb0; kb < kb0 + k_blocks; ++kb, ++it) {
                     const int s = it % NS;
                     const uint32_t ph = (it / NS) & 1u;
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, p.status, abort_flag)) { ok = false; break; }
+                    // test hook: the stage is never loaded nor announced, so the MMA warp's wait for it runs out
+                    if (p.skip_last_stage && unit + num_pairs >= num_units && kb == kb0 + k_blocks - 1) break;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, wc)) { ok = false; break; }
                     const uint32_t lead_full = map_to_cta(full_bar(s), 0);
                     if (leader) mbar_arrive_expect_tx(full_bar(s), STAGE_TX);
                     const uint32_t a_dst = smem_base + s * C::STAGE;
@@ -424,7 +434,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             for (int unit = pair; unit < num_units && ok; unit += num_pairs, ++local_tile) {
                 const int k_blocks = decode(unit).k_blocks;
                 const uint32_t buf = local_tile % NB, use = local_tile / NB;
-                if (!mbar_wait(acc_empty_bar(buf), (use & 1u) ^ 1u, p.status, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(acc_empty_bar(buf), (use & 1u) ^ 1u, wc)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {     // stage index inside the unit's K range
@@ -437,13 +447,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         const int atom0 = kb * ATOMS_PER_STAGE;
                         const uint32_t region = group_it % META_REGIONS;
                         if ((atom0 & 3) == 0 &&
-                            !mbar_wait(meta_full_bar(region), (group_it / META_REGIONS) & 1u, p.status, abort_flag)) {
+                            !mbar_wait(meta_full_bar(region), (group_it / META_REGIONS) & 1u, wc)) {
                             ok = false;
                             break;
                         }
                         meta_cols = tmem_base + C::META_COL0 + 16 * region + 4 * (atom0 & 3);
                     }
-                    if (!mbar_wait(full_bar(s), ph, p.status, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(s), ph, wc)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_src = smem_base + s * C::STAGE;
                     const uint32_t b_src = a_src + C::A_STAGE;
@@ -502,7 +512,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint32_t buf = local_tile % NB, use = local_tile / NB;
             const uint32_t acc_base = lane_base + buf * BN;
             const uint32_t lead_acc_empty = map_to_cta(acc_empty_bar(buf), 0);
-            if (!epilogue_all(mbar_wait_warp(acc_full_bar(buf), use & 1u, p.status, abort_flag))) { ok = false; break; }
+            if (!epilogue_all(mbar_wait_warp(acc_full_bar(buf), use & 1u, wc))) { ok = false; break; }
             tc_fence_after();
             if (OUT_F32) {
 #pragma unroll 1
@@ -708,7 +718,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint32_t group_it = 0;
         while (h0) {
             const uint32_t region = group_it % META_REGIONS;
-            if (!mbar_wait_warp(meta_empty_bar(region), ((group_it / META_REGIONS) & 1u) ^ 1u, p.status, abort_flag)) break;
+            if (!mbar_wait_warp(meta_empty_bar(region), ((group_it / META_REGIONS) & 1u) ^ 1u, wc)) break;
             tc_fence_after();
 #pragma unroll
             for (int i = 0; i < 4; ++i) tmem_st_32x4(lane_base + 16 * region + 4 * i, q0[i]);
@@ -807,7 +817,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         while (h0) {
             const int s = it % NS;
             const uint32_t ph = (it / NS) & 1u;
-            if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, p.status, abort_flag)) break;
+            if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, wc)) break;
             uint8_t *b_dst = ring + s * C::STAGE + C::A_STAGE + (seg >> 2) * (BK * 128);
             const int j0 = (seg & 3) * 2;
 #pragma unroll
@@ -940,6 +950,8 @@ struct DeviceOnce {
     }
 };
 
+int g_inject_stall = 0;   // test hook: see sste_debug_inject_stall
+
 struct SplitPlan { int splits, split_from; };
 SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn);
 
@@ -979,6 +991,15 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         return SSTE_ERR_CUDA;
     const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM), n_tiles = (p.N + BN - 1) / BN;
     GemmParams pp = p;
+    pp.wait_limit_ns = WAIT_LIMIT_NS;
+    pp.skip_last_stage = 0;
+    if (g_inject_stall) {
+        // Test hook (sste_debug_inject_stall): only a dense product of ONE output tile takes the fault, so that
+        // exactly one CTA pair runs into the expired wait; every other launch refuses while the hook is armed.
+        if (SPARSE || BCOMP || OUT_F32 || m_tiles * n_tiles != 1) return SSTE_ERR_INVALID_ARG;
+        pp.wait_limit_ns = 1000000ull;      // one millisecond
+        pp.skip_last_stage = 1;
+    }
     if (BCOMP) pp.b_vals = static_cast<const uint8_t *>(B);
     if (pp.out_amax && cudaMemsetAsync(pp.out_amax, 0, sizeof(unsigned int), stream) != cudaSuccess) return SSTE_ERR_CUDA;
     const int tiles = m_tiles * n_tiles;
@@ -1013,6 +1034,7 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
 }
 
 int g_force_splits = 0;   // test hook: 0 = automatic split-K factor
+
 
 // Split-K plan.  Tiles that fill complete waves of CTA pairs are computed whole; the tiles of the last,
 // partial wave (all of them when there are fewer tiles than pairs, as for the weight gradient of a
@@ -1120,6 +1142,11 @@ extern "C" sste_status sste_debug_force_splits(int splits)
 {
     if (splits < 0 || splits > 4) return SSTE_ERR_INVALID_ARG;
     g_force_splits = splits;
+    return SSTE_OK;
+}
+extern "C" sste_status sste_debug_inject_stall(int on)
+{
+    g_inject_stall = on ? 1 : 0;
     return SSTE_OK;
 }
 extern "C" sste_status sste_debug_force_tile_width(int bn)
