@@ -386,6 +386,11 @@ def measure_config(cfg_id, args, env, full):
     value = world * flops_step / (ms_per_step * 1e-3) / 1e12
     clocks = sampler.window(t_host0, t_host1)
 
+    if args.timed_only:        # a profiler run: the warm-up and the timed steps only
+        ctx.close()
+        return {"value": value, "unit": UNIT, "ms_per_step": ms_per_step, "repeats": repeats, "timed_only": True,
+                "dtype": "fp8" if fp8 else "bf16", "config": workload_config(cfg_id, cfg, world), "clocks": clocks}
+
     # ---- sustained: graph replays back to back for two seconds, no flush, no host gaps: what a training loop sees
     sustained = None
     if graph is not None:
@@ -585,7 +590,7 @@ def run_gpu(args):
 
     main = measure_config(args.config, args, env, full=True)
     per_config = {}
-    if world == 1 and not args.no_per_config:
+    if world == 1 and not args.no_per_config and not args.timed_only:
         for other in (2, 3):
             if other != args.config:
                 r = measure_config(other, args, env, full=False)
@@ -595,7 +600,9 @@ def run_gpu(args):
                                                             "rooflines", "kernels", "launches_per_step")}
     sampler.stop()
 
-    if rank == 0:
+    if rank == 0 and args.timed_only:
+        print(json.dumps(main), flush=True)
+    elif rank == 0:
         cpu_tokens = args.ref_tokens or oracle_tokens(args.config, 1.0e12)
         cpu_base, _ = time_oracle(args.config, cpu_tokens, 3, 1)
         line = {
@@ -680,6 +687,8 @@ def main():
                     help="run grad_W and grad_X back to back instead of grad_W on a side stream beside grad_X")
     ap.add_argument("--no-graph", action="store_true", help="launch the timed steps eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-per-config", action="store_true", help="measure only --config, not the other bf16 workloads")
+    ap.add_argument("--timed-only", action="store_true",
+                    help="stop after the timed steps (for profiler runs: few launches, no end-to-end / CPU legs)")
     ap.add_argument("--min-timed-ms", type=float, default=1000.0, help="repeat the K timed steps until this much is timed")
     ap.add_argument("--sustained-ms", type=float, default=2000.0, help="length of the back-to-back sustained loop")
     ap.add_argument("--ref-tokens", type=int, default=0, help="tokens per layer in the CPU-oracle sample (0 = sized to a budget)")

@@ -330,6 +330,12 @@ sste_status sste_debug_force_tile_width(int bn);
  * falls back to the automatic choice. */
 sste_status sste_debug_force_splits(int splits);
 
+/* The products hand their output tiles to the CTA pairs band by band (a band = group_m consecutive rows of
+ * 256-row tiles, row index fastest inside a band), with group_m chosen from the operand sizes so that operands
+ * are read from HBM about once.  This hook pins group_m (0 = automatic; values above the number of tile rows mean
+ * plain column-major order) so that tests can cover every order. */
+sste_status sste_debug_force_tile_order(int group_m);
+
 /* Test hook for the bounded waits.  While armed (on != 0), a dense sste_linear_bwd_input (Wt_dense given, bf16
  * output) whose output is ONE tile (T <= 256, I <= 256) leaves the last K stage of its operand pipeline unloaded
  * and limits every device-side wait to one millisecond instead of two seconds: the wait for that stage runs out,

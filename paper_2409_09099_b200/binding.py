@@ -31,6 +31,7 @@ EXPORTS = [
     "sste_workspace_bytes_recommended", "sste_beta_init_static", "sste_debug_launch_count", "sste_flip_count",
     "sste_project_compress_variant", "sste_beta_init_l1", "sste_srste_decay", "sste_project_amax",
     "sste_decompress", "sste_padded_dim", "sste_pad_2d", "sste_crop_2d", "sste_debug_inject_stall",
+    "sste_debug_force_tile_order",
 ]
 
 
@@ -238,6 +239,9 @@ class Context:
 
     def debug_force_splits(self, splits: int):
         self._check(self.lib.sste_debug_force_splits(splits))
+
+    def debug_force_tile_order(self, group_m: int):
+        self._check(self.lib.sste_debug_force_tile_order(group_m))
 
     def debug_inject_stall(self, on: bool):
         self._check(self.lib.sste_debug_inject_stall(1 if on else 0))

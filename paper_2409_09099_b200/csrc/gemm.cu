@@ -241,6 +241,22 @@ __host__ __device__ constexpr uint32_t instr_desc(bool sparse, uint32_t afmt, ui
 
 // ------------------------------------------------------------------ kernel
 
+// Order in which output tiles are handed to the CTA pairs (pair p takes tiles p, p + pairs, ...).  Tiles are
+// numbered band by band: a band is `group_m` consecutive rows of tiles, and inside a band the row index runs
+// fastest.  The 74 tiles in flight at any time therefore cover group_m tile rows x 74 / group_m tile columns,
+// and the A rows of a band stay in L2 while the band sweeps over all of B.  group_m = m_tiles is plain
+// column-major order (all of A resident, B streamed once).
+__host__ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int group_m, int &mt, int &nt)
+{
+    const int per_band = group_m * n_tiles;
+    const int band = tile / per_band;
+    const int first = band * group_m;
+    const int rows = (m_tiles - first < group_m) ? (m_tiles - first) : group_m;
+    const int within = tile - band * per_band;
+    mt = first + within % rows;
+    nt = within / rows;
+}
+
 struct GemmParams {
     int M, N, K;            // logical problem: D[M, N] = A[M, K] * B
     void *D;                // output (used by the direct-store fp32 epilogue)
@@ -254,6 +270,7 @@ struct GemmParams {
     const uint8_t *b_vals;  // compressed-B kernels: the 2:4 values of B [K, N/2]; its metadata image is `meta`
     unsigned long long wait_limit_ns;   // limit of every device-side wait
     int skip_last_stage;    // stall-injection test hook: the producer leaves the last K stage of the launch unloaded
+    int group_m;            // tile rows per band of the tile order (see tile_coords)
     int splits;             // split-K factor of the tiles from `split_from` on (1 = none)
     int split_from;         // first split tile: tiles below it are computed whole
     float *partials;        // split-K: fp32 partial tiles [tile][cta][split][128][BN], summed by splitk_reduce_kernel
@@ -395,7 +412,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             for (int unit = pair; unit < num_units && ok; unit += num_pairs) {
                 const Unit u = decode(unit);
                 const int tile = u.tile, k_blocks = u.k_blocks, kb0 = u.split * u.k_blocks;
-                const int mt = tile % m_tiles, nt = tile / m_tiles;
+                int mt, nt;
+                tile_coords(tile, m_tiles, n_tiles, p.group_m, mt, nt);
                 const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;      // this CTA's rows of A
                 const int n0 = nt * BN + static_cast<int>(rank) * (BN / 2);    // this CTA's half of B
                 for (int kb = kb0; kb < kb0 + k_blocks; ++kb, ++it) {
@@ -506,7 +524,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         for (int unit = pair; unit < num_units && ok; unit += num_pairs, ++local_tile) {
             const Unit u = decode(unit);
             const int tile = u.tile, split = u.split;
-            const int mt = tile % m_tiles, nt = tile / m_tiles;
+            int mt, nt;
+            tile_coords(tile, m_tiles, n_tiles, p.group_m, mt, nt);
             const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;
             const int n0 = nt * BN;
             const uint32_t buf = local_tile % NB, use = local_tile / NB;
@@ -693,7 +712,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         auto l_setup = [&]() {
             if (l_unit >= num_units) return;
             const Unit u = decode(l_unit);
-            const int m0 = (u.tile % m_tiles) * 2 * BM + static_cast<int>(rank) * BM;
+            int mt, nt;
+            tile_coords(u.tile, m_tiles, n_tiles, p.group_m, mt, nt);
+            const int m0 = mt * 2 * BM + static_cast<int>(rank) * BM;
             l_rows = m0 < p.M;
             l_src = reinterpret_cast<const uint4 *>(meta + static_cast<size_t>(m0 / BM) * k_atoms * 2048) + quarter * 32 + lane;
             l_a0 = u.split * u.k_blocks * ATOMS_PER_STAGE;
@@ -778,7 +799,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         auto e_setup = [&]() {
             if (e_unit >= num_units) return;
             const Unit u = decode(e_unit);
-            const int n0 = (u.tile / m_tiles) * BN + static_cast<int>(rank) * (BN / 2);
+            int mt, nt;
+            tile_coords(u.tile, m_tiles, n_tiles, p.group_m, mt, nt);
+            const int n0 = nt * BN + static_cast<int>(rank) * (BN / 2);
             e_cols = n0 < p.N;
             e_vals = p.b_vals + (static_cast<size_t>(n0 / 2) + seg * (EPU / 2)) * ELT + r0 * row_bytes;
             e_meta = meta + static_cast<size_t>(n0 >> 7) * 2048;
@@ -890,7 +913,8 @@ bool make_map(const sste_ctx *ctx, CUtensorMap *map, const void *base, int elt, 
 // Split-K second pass over the split tiles: out[m, n] = bf16(scale * sum over splits, in split order, of
 // the fp32 partial tiles [split tile][cta][split][128][bn]).  One thread per 8 consecutive n.
 __global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, int splits, int m_tiles, int split_from,
+splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, int splits, int m_tiles, int n_tiles,
+                     int group_m, int split_from,
                      int n_split_tiles, const float *__restrict__ a_amax, float a_fp8_max,
                      const float *__restrict__ b_amax, float b_fp8_max, unsigned int *__restrict__ out_amax,
                      uint4 *__restrict__ out)
@@ -906,8 +930,10 @@ splitk_reduce_kernel(const float *__restrict__ partials, int M, int N, int bn, i
         const int row = static_cast<int>((v / vec_per_row) % BM);
         const size_t slot = v / (static_cast<size_t>(vec_per_row) * BM);        // (split tile, cta)
         const int tile = split_from + static_cast<int>(slot >> 1);
-        const int m = (tile % m_tiles) * 2 * BM + static_cast<int>(slot & 1) * BM + row;
-        const int n = (tile / m_tiles) * bn + col;
+        int mt, nt;
+        tile_coords(tile, m_tiles, n_tiles, group_m, mt, nt);
+        const int m = mt * 2 * BM + static_cast<int>(slot & 1) * BM + row;
+        const int n = nt * bn + col;
         if (m >= M || n >= N) continue;
         const float *src = partials + (slot * splits * BM + row) * bn + col;
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -951,6 +977,25 @@ struct DeviceOnce {
 };
 
 int g_inject_stall = 0;   // test hook: see sste_debug_inject_stall
+int g_force_group_m = 0;  // test hook: 0 = automatic band height of the tile order
+
+// Band height of the tile order from the operand sizes (a_tile / b_tile: bytes of one tile row of A / one tile
+// column of B over the whole reduction).  L2 is 126 MB; an operand that takes less than half of it stays
+// resident whatever the order.
+//   A small: plain column-major order (every pair of a wave shares a few columns of B, B is read once).
+//   else:    bands of about sqrt(pairs * b_tile / a_tile) tile rows: a wave then loads the least bytes, the band's
+//            A rows are read once while B, if it fits, stays in L2 across bands.
+int pick_group_m(int m_tiles, int n_tiles, int pairs, double a_tile, double b_tile)
+{
+    if (g_force_group_m > 0) return g_force_group_m < m_tiles ? g_force_group_m : m_tiles;
+    const double l2_budget = 56e6;
+    if (a_tile * m_tiles <= l2_budget || m_tiles <= 1 || n_tiles <= 1) return m_tiles;
+    double g = __builtin_sqrt(static_cast<double>(pairs) * b_tile / a_tile);
+    int gm = static_cast<int>(g + 0.5);
+    if (gm < 1) gm = 1;
+    if (gm > m_tiles) gm = m_tiles;
+    return gm;
+}
 
 struct SplitPlan { int splits, split_from; };
 SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn);
@@ -1001,6 +1046,9 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         pp.skip_last_stage = 1;
     }
     if (BCOMP) pp.b_vals = static_cast<const uint8_t *>(B);
+    pp.group_m = pick_group_m(m_tiles, n_tiles, ctx->sm_count / 2,
+                              static_cast<double>(p.K) * (SPARSE ? 0.5 * ELT + 0.125 : 1.0 * ELT) * 2 * BM,
+                              static_cast<double>(p.K) * ((BCOMP ? 0.5 : 1.0) * ELT) * BN);
     if (pp.out_amax && cudaMemsetAsync(pp.out_amax, 0, sizeof(unsigned int), stream) != cudaSuccess) return SSTE_ERR_CUDA;
     const int tiles = m_tiles * n_tiles;
     SplitPlan plan{1, tiles};
@@ -1024,7 +1072,7 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         size_t blocks = (vecs + 255) / 256;
         if (blocks > static_cast<size_t>(ctx->sm_count) * 16) blocks = static_cast<size_t>(ctx->sm_count) * 16;
         if (sste_launch(splitk_reduce_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(256), 0, stream,
-                        pp.partials, p.M, p.N, BN, pp.splits, m_tiles, pp.split_from, n_split_tiles, p.a_amax,
+                        pp.partials, p.M, p.N, BN, pp.splits, m_tiles, n_tiles, pp.group_m, pp.split_from, n_split_tiles, p.a_amax,
                         p.a_fp8_max, p.b_amax, p.b_fp8_max, pp.out_amax, static_cast<uint4 *>(p.D)) != cudaSuccess)
             return SSTE_ERR_CUDA;
     }
@@ -1142,6 +1190,12 @@ extern "C" sste_status sste_debug_force_splits(int splits)
 {
     if (splits < 0 || splits > 4) return SSTE_ERR_INVALID_ARG;
     g_force_splits = splits;
+    return SSTE_OK;
+}
+extern "C" sste_status sste_debug_force_tile_order(int group_m)
+{
+    if (group_m < 0) return SSTE_ERR_INVALID_ARG;
+    g_force_group_m = group_m;
     return SSTE_OK;
 }
 extern "C" sste_status sste_debug_inject_stall(int on)

@@ -310,3 +310,51 @@ def test_overlapped_backward_equals_serial(ctx, fp8):
         assert side_ctx.poll_device_status() == 0
     finally:
         side_ctx.close()
+
+
+@pytest.mark.parametrize("group_m", [1, 2, 3, 1000])
+def test_tile_order_does_not_change_the_products(ctx, group_m):
+    """Every band height of the tile order (incl. a last, partial band and split tail tiles) gives the same bits."""
+    O, I, T = 1280, 768, 1792                      # forward 5 x 7, grad_W 5 x 3, grad_X 7 x 3 tiles of 256 x 256
+    W, X, dY = synth.gaussian_bf16(91, (O, I), 0.02), synth.gaussian_bf16(92, (T, I), 1.0), synth.gaussian_bf16(93, (T, O), 1e-2)
+    Wd, Xd, dYd = dbf16(W), dbf16(X), dbf16(dY)
+    beta_dev = torch.zeros(1, dtype=torch.float32, device=DEV)
+    ctx.beta_init(Wd, beta_dev)
+    vals, meta = ctx.alloc_compressed(O, I)
+    dense = torch.empty((O, I), dtype=torch.bfloat16, device=DEV)
+    ctx.project_compress(Wd, beta_dev, vals, meta, dense)
+    gvals, gmeta = ctx.alloc_compressed(O, T)
+    ctx.mvue_sparsify(dYd, 7, 1, 0, gvals, gmeta)
+
+    def run():
+        Y = torch.empty((T, O), dtype=torch.bfloat16, device=DEV)
+        dW = torch.empty((O, I), dtype=torch.bfloat16, device=DEV)
+        dX = torch.empty((T, I), dtype=torch.bfloat16, device=DEV)
+        dXc = torch.empty((T, I), dtype=torch.bfloat16, device=DEV)
+        ctx.linear_fwd(Xd, vals, meta, Y)
+        ctx.linear_bwd_weight(gvals, gmeta, Xd, dW)
+        ctx.linear_bwd_input(dYd, dense, dX)
+        ctx.linear_bwd_input(dYd, None, dXc, vals=vals, meta=meta)
+        torch.cuda.synchronize()
+        return Y, dW, dX, dXc
+
+    # the same split plan on both sides: the order of the tiles must not change a single bit
+    results = {}
+    try:
+        for splits in (1, 2):
+            ctx.debug_force_splits(splits)
+            for order in (1000, group_m):
+                ctx.debug_force_tile_order(order)
+                results[splits, order] = run()
+    finally:
+        ctx.debug_force_splits(0)
+        ctx.debug_force_tile_order(0)
+    for splits in (1, 2):
+        for a, b in zip(results[splits, 1000], results[splits, group_m]):
+            assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    refs = (orc.linear_fwd(X, orc.BF16, bits16(vals), canonical_meta(ctx, meta, O, I, 0), orc.BF16),
+            orc.linear_bwd_weight(bits16(gvals), canonical_meta(ctx, gmeta, O, T, 0), orc.BF16, X, orc.BF16),
+            orc.linear_bwd_input(dY, orc.BF16, bits16(dense), orc.BF16))
+    for a, ref in zip(results[2, group_m][:3], refs):
+        assert rel_fro(a.float().cpu().numpy(), ref) <= BF16_GEMM_TOL
+    assert ctx.poll_device_status() == 0
