@@ -17,6 +17,7 @@
 #include <cuda.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -515,6 +516,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int row = quarter * 32 + lane;           // row of this CTA's 128 x BN accumulator
         const float scale = sste_out_scale(p.a_amax, p.a_fp8_max, p.b_amax, p.b_fp8_max);
         const bool want_amax = (p.out_amax != nullptr);
+        const bool plain = !want_amax && scale == 1.0f;
         uint32_t amax2 = 0;                            // bf16 output: running max of the magnitude bits, two lanes of 16
         float amaxf = 0.0f;                            // fp32 output
         const bool store_thread = (threadIdx.x == 64);
@@ -599,17 +601,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             }
             // bf16 output in panels of PANEL columns through two 16 KB staging buffers and TMA stores.
             // 32 accumulator columns -> bf16 -> staging buffer `sb`, columns [c0, c0 + 32) of the panel
-            auto stage_chunk = [&](const uint32_t (&r)[32], uint8_t *sb, int c0) {
+            // Two accumulator values -> one word of two bf16 (packed conversion).  PLAIN: unit scale and no amax
+            // wanted (every bf16 product of the path): no multiply, no maximum.
+            auto pack2 = [&](uint32_t a, uint32_t b, auto plain_tag) -> uint32_t {
+                float lo = __uint_as_float(a), hi = __uint_as_float(b);
+                if (!decltype(plain_tag)::value) {
+                    lo = __fmul_rn(lo, scale);
+                    hi = __fmul_rn(hi, scale);
+                }
+                const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+                const uint32_t w = *reinterpret_cast<const uint32_t *>(&v);
+                if (!decltype(plain_tag)::value) amax2 = __vmaxu2(amax2, w & 0x7fff7fffu);
+                return w;
+            };
+            auto stage_impl = [&](const uint32_t (&r)[32], uint8_t *sb, int c0, auto plain_tag) {
                 if (OUT_T) {
                     // staging[n][m]: PANEL rows of 128 bf16; a warp writes 32 consecutive m per n
                     uint16_t *st = reinterpret_cast<uint16_t *>(sb);
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
-                        const uint32_t lo = sste_f32_to_bf16_bits(__fmul_rn(__uint_as_float(r[c]), scale));
-                        const uint32_t hi = sste_f32_to_bf16_bits(__fmul_rn(__uint_as_float(r[c + 1]), scale));
-                        st[(c0 + c) * BM + row] = static_cast<uint16_t>(lo);
-                        st[(c0 + c + 1) * BM + row] = static_cast<uint16_t>(hi);
-                        if (want_amax) amax2 = __vmaxu2(amax2, (lo | (hi << 16)) & 0x7fff7fffu);
+                        const uint32_t w = pack2(r[c], r[c + 1], plain_tag);
+                        st[(c0 + c) * BM + row] = static_cast<uint16_t>(w);
+                        st[(c0 + c + 1) * BM + row] = static_cast<uint16_t>(w >> 16);
                     }
                 } else {
                     // [128 rows][64 bf16] with the 128-byte swizzle of the TMA store: 16-byte chunk index ^= row & 7
@@ -619,15 +632,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     for (int c = 0; c < 4; ++c) {
                         uint32_t w[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float lo = __fmul_rn(__uint_as_float(r[8 * c + 2 * e]), scale);
-                            const float hi = __fmul_rn(__uint_as_float(r[8 * c + 2 * e + 1]), scale);
-                            w[e] = sste_f32_to_bf16_bits(lo) | (sste_f32_to_bf16_bits(hi) << 16);
-                            if (want_amax) amax2 = __vmaxu2(amax2, w[e] & 0x7fff7fffu);
-                        }
+                        for (int e = 0; e < 4; ++e) w[e] = pack2(r[8 * c + 2 * e], r[8 * c + 2 * e + 1], plain_tag);
                         *reinterpret_cast<uint4 *>(dst + (((chunk0 + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
+            };
+            auto stage_chunk = [&](const uint32_t (&r)[32], uint8_t *sb, int c0) {
+                if (plain) stage_impl(r, sb, c0, std::true_type{});
+                else stage_impl(r, sb, c0, std::false_type{});
             };
             // staging buffer of the next panel becomes writable once the store issued two panels ago has read it
             auto acquire_staging = [&]() -> uint32_t {
