@@ -1010,7 +1010,7 @@ int pick_group_m(int m_tiles, int n_tiles, int pairs, double a_tile, double b_ti
 }
 
 struct SplitPlan { int splits, split_from; };
-SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn);
+SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn, double stage_us);
 
 template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32, bool BCOMP = false>
 sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void *meta, const GemmParams &p,
@@ -1064,7 +1064,8 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
     if (pp.out_amax && cudaMemsetAsync(pp.out_amax, 0, sizeof(unsigned int), stream) != cudaSuccess) return SSTE_ERR_CUDA;
     const int tiles = m_tiles * n_tiles;
     SplitPlan plan{1, tiles};
-    if (!OUT_F32 && !OUT_T) plan = pick_split_plan(ctx, tiles, (p.K + BK - 1) / BK, SPARSE ? 4 / (BK / 128) : 1, BN);
+    if (!OUT_F32 && !OUT_T)   // a stage takes about 790 clk (sparse) / 512 clk (dense) at 1.9 GHz
+        plan = pick_split_plan(ctx, tiles, (p.K + BK - 1) / BK, SPARSE ? 4 / (BK / 128) : 1, BN, SPARSE ? 0.42 : 0.27);
     pp.splits = plan.splits;
     pp.split_from = plan.split_from;
     pp.partials = ctx->splitk_partials;
@@ -1100,7 +1101,7 @@ int g_force_splits = 0;   // test hook: 0 = automatic split-K factor
 // partial wave (all of them when there are fewer tiles than pairs, as for the weight gradient of a
 // GPT-2-sized layer: 36 tiles, 74 pairs) are cut into `splits` K ranges so that the wave takes 1/splits
 // of a tile time.  `align` = stages per metadata group (K ranges must start on a group boundary).
-SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn)
+SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn, double stage_us)
 {
     SplitPlan none{1, tiles};
     if (!ctx->splitk_partials) return none;
@@ -1109,13 +1110,15 @@ SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int alig
     const int tail = tiles - whole;
     if (tail == 0) return none;
     int best = 1;
-    double best_cost = 1.0;            // time of the last wave in units of one whole tile
+    const double tile_us = k_blocks * stage_us;
+    double best_cost = tile_us;        // time of the last wave, microseconds
     for (int s = 2; s <= 4; ++s) {
         if (k_blocks % (s * align) != 0 || k_blocks / s < 8) continue;
         if (static_cast<size_t>(tail) * 2 * s * BM * bn * sizeof(float) > ctx->splitk_partial_bytes) continue;
         if (g_force_splits == s) return SplitPlan{s, whole};
         const int waves = (tail * s + pairs - 1) / pairs;
-        const double cost = static_cast<double>(waves) / s + 0.08 * s;   // + partial tiles' round trip
+        // + the second pass (a launch of its own) and the partial tiles' round trip through L2
+        const double cost = tile_us * waves / s + 4.0 + 0.3 * s;
         if (cost < best_cost - 1e-9) { best = s; best_cost = cost; }
     }
     if (g_force_splits == 1 || best == 1) return none;
