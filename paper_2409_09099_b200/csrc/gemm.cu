@@ -277,11 +277,16 @@ struct GemmParams {
     float *partials;        // split-K: fp32 partial tiles [tile][cta][split][128][BN], summed by splitk_reduce_kernel
 };
 
-// 32 lanes x 4 consecutive 32-bit columns <- 4 registers per thread
-__device__ __forceinline__ void tmem_st_32x4(uint32_t taddr, uint4 v)
+// 32 lanes x 16 consecutive 32-bit columns <- 16 registers per thread (four metadata atoms in one instruction)
+__device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint4 (&v)[4])
 {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
-                 ::"r"(taddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0].x), "r"(v[0].y), "r"(v[0].z), "r"(v[0].w), "r"(v[1].x), "r"(v[1].y), "r"(v[1].z),
+          "r"(v[1].w), "r"(v[2].x), "r"(v[2].y), "r"(v[2].z), "r"(v[2].w), "r"(v[3].x), "r"(v[3].y), "r"(v[3].z),
+          "r"(v[3].w)
+        : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -712,9 +717,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // ------------------------------------------------------------ metadata warps (6..9, both CTAs)
         // HBM -> registers -> tensor memory: lane L of an atom's image is exactly the 16 bytes the
         // instruction expects in tensor-memory lane L, four 32-bit columns per atom.
-        // The loads run three groups (of four atoms) ahead of the stores, in registers: a group's round trip
+        // The loads run six groups (of four atoms) ahead of the stores, in registers: a group's round trip
         // to L2 / HBM is then off the path that feeds the MMA warp (with load -> store -> signal in sequence
-        // per group, that latency, not the tensor pipe, set the pace of every sparse product).
+        // per group, that latency, not the tensor pipe, set the pace of every sparse product; with three groups
+        // in flight the 8-bit kinds, which consume two atoms per stage, were still paced by it).
         const int quarter = warp & 3;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + C::META_COL0;
         // loader cursor: (unit, first atom of the next group)
@@ -746,25 +752,31 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             return true;
         };
         l_setup();
-        uint4 q0[4], q1[4], q2[4];
-        bool h0 = l_issue(q0), h1 = l_issue(q1), h2 = l_issue(q2);
+        // META_DEPTH groups of loads are in flight per lane (a ring of registers; the loop is unrolled over it):
+        // a group must be on its way for several stages before its turn, or the round trip to L2 paces the warp
+        constexpr int META_DEPTH = 6;
+        uint4 q[META_DEPTH][4];
+        bool have[META_DEPTH];
+#pragma unroll
+        for (int d = 0; d < META_DEPTH; ++d) have[d] = l_issue(q[d]);
         uint32_t group_it = 0;
-        while (h0) {
-            const uint32_t region = group_it % META_REGIONS;
-            if (!mbar_wait_warp(meta_empty_bar(region), ((group_it / META_REGIONS) & 1u) ^ 1u, wc)) break;
-            tc_fence_after();
+        bool running = true;
+        while (running) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) tmem_st_32x4(lane_base + 16 * region + 4 * i, q0[i]);
-            tmem_st_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(meta_full_bar(region), 0));
-            ++group_it;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { q0[i] = q1[i]; q1[i] = q2[i]; }
-            h0 = h1;
-            h1 = h2;
-            h2 = l_issue(q2);
+            for (int d = 0; d < META_DEPTH; ++d) {
+                if (!running) break;
+                if (!have[d]) { running = false; break; }
+                const uint32_t region = group_it % META_REGIONS;
+                if (!mbar_wait_warp(meta_empty_bar(region), ((group_it / META_REGIONS) & 1u) ^ 1u, wc)) { running = false; break; }
+                tc_fence_after();
+                tmem_st_32x16(lane_base + 16 * region, q[d]);      // one store for the group's four atoms
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(meta_full_bar(region), 0));
+                ++group_it;
+                have[d] = l_issue(q[d]);
+            }
         }
     } else if (BCOMP) {
         // ------------------------------------------------------------ expander warps (6..9, both CTAs)
