@@ -336,6 +336,15 @@ sste_status sste_debug_force_splits(int splits);
  * plain column-major order) so that tests can cover every order. */
 sste_status sste_debug_force_tile_order(int group_m);
 
+/* What the library would decide for a product launch, computed on the host (no device is touched): product 0 =
+ * sste_linear_fwd, 1 = sste_linear_bwd_weight, 2 = sste_linear_bwd_input (dense operand), operands of dtype opdt,
+ * bf16 output, on a GPU of sm_count SMs with a context workspace of workspace_bytes.  Outputs (each nullable): the
+ * tile width, the split-K factor and the first split tile, the band height of the tile order.  The debug hooks
+ * above apply.  sste_debug_tile_coords maps a tile number to its (row, column) of tiles under a band height. */
+sste_status sste_debug_plan(int product, sste_dtype opdt, int O, int I, int T, int sm_count, size_t workspace_bytes,
+                            int *tile_width, int *splits, int *split_from, int *group_m);
+sste_status sste_debug_tile_coords(int tile, int m_tiles, int n_tiles, int group_m, int *mt, int *nt);
+
 /* Test hook for the bounded waits.  While armed (on != 0), a dense sste_linear_bwd_input (Wt_dense given, bf16
  * output) whose output is ONE tile (T <= 256, I <= 256) leaves the last K stage of its operand pipeline unloaded
  * and limits every device-side wait to one millisecond instead of two seconds: the wait for that stage runs out,

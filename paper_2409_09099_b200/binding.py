@@ -31,7 +31,7 @@ EXPORTS = [
     "sste_workspace_bytes_recommended", "sste_beta_init_static", "sste_debug_launch_count", "sste_flip_count",
     "sste_project_compress_variant", "sste_beta_init_l1", "sste_srste_decay", "sste_project_amax",
     "sste_decompress", "sste_padded_dim", "sste_pad_2d", "sste_crop_2d", "sste_debug_inject_stall",
-    "sste_debug_force_tile_order",
+    "sste_debug_force_tile_order", "sste_debug_plan", "sste_debug_tile_coords",
 ]
 
 
@@ -74,6 +74,17 @@ def _stream():
 def padded_dim(n: int) -> int:
     """sste_padded_dim: the next multiple of 128."""
     return int(load().sste_padded_dim(n))
+
+
+def plan(product: int, opdt: int, O: int, I: int, T: int, sm_count: int = 148, workspace_bytes: int | None = None):
+    """sste_debug_plan: (tile width, split-K factor, first split tile, band height) of a product launch; host only."""
+    lib = load()
+    ws = lib.sste_workspace_bytes_recommended() if workspace_bytes is None else workspace_bytes
+    out = [ctypes.c_int() for _ in range(4)]
+    st = lib.sste_debug_plan(product, opdt, O, I, T, sm_count, ctypes.c_size_t(ws), *[ctypes.byref(o) for o in out])
+    if st != OK:
+        raise SsteError(st, lib.sste_status_string(st).decode())
+    return tuple(o.value for o in out)
 
 
 def launch_count() -> int:

@@ -1022,7 +1022,27 @@ int pick_group_m(int m_tiles, int n_tiles, int pairs, double a_tile, double b_ti
 }
 
 struct SplitPlan { int splits, split_from; };
-SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn, double stage_us);
+SplitPlan pick_split_plan(int sm_count, size_t partial_bytes, int tiles, int k_blocks, int align, int bn, double stage_us);
+
+// Everything the host decides about one product launch of a given tile width (the width itself: pick_bn).
+struct LaunchPlan { int splits, split_from, group_m; };
+LaunchPlan make_plan(bool sparse, int elt, int bn, bool out_t, bool out_f32, bool bcomp, int sm_count,
+                     size_t partial_bytes, int M, int N, int K)
+{
+    const int bk = (sparse ? 256 : 128) / elt;
+    const int m_tiles = (M + 2 * BM - 1) / (2 * BM), n_tiles = (N + bn - 1) / bn, tiles = m_tiles * n_tiles;
+    LaunchPlan plan{1, tiles, m_tiles};
+    plan.group_m = pick_group_m(m_tiles, n_tiles, sm_count / 2,
+                                static_cast<double>(K) * (sparse ? 0.5 * elt + 0.125 : 1.0 * elt) * 2 * BM,
+                                static_cast<double>(K) * ((bcomp ? 0.5 : 1.0) * elt) * bn);
+    if (!out_f32 && !out_t) {   // a stage takes about 790 clk (sparse) / 512 clk (dense) at 1.9 GHz
+        const SplitPlan sp = pick_split_plan(sm_count, partial_bytes, tiles, (K + bk - 1) / bk, sparse ? 4 / (bk / 128) : 1,
+                                             bn, sparse ? 0.42 : 0.27);
+        plan.splits = sp.splits;
+        plan.split_from = sp.split_from;
+    }
+    return plan;
+}
 
 template <bool SPARSE, BMajor BMAJ, int ELT, int BN, bool OUT_T, bool OUT_F32, bool BCOMP = false>
 sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void *meta, const GemmParams &p,
@@ -1070,14 +1090,11 @@ sste_status launch(const sste_ctx *ctx, const void *A, const void *B, const void
         pp.skip_last_stage = 1;
     }
     if (BCOMP) pp.b_vals = static_cast<const uint8_t *>(B);
-    pp.group_m = pick_group_m(m_tiles, n_tiles, ctx->sm_count / 2,
-                              static_cast<double>(p.K) * (SPARSE ? 0.5 * ELT + 0.125 : 1.0 * ELT) * 2 * BM,
-                              static_cast<double>(p.K) * ((BCOMP ? 0.5 : 1.0) * ELT) * BN);
     if (pp.out_amax && cudaMemsetAsync(pp.out_amax, 0, sizeof(unsigned int), stream) != cudaSuccess) return SSTE_ERR_CUDA;
     const int tiles = m_tiles * n_tiles;
-    SplitPlan plan{1, tiles};
-    if (!OUT_F32 && !OUT_T)   // a stage takes about 790 clk (sparse) / 512 clk (dense) at 1.9 GHz
-        plan = pick_split_plan(ctx, tiles, (p.K + BK - 1) / BK, SPARSE ? 4 / (BK / 128) : 1, BN, SPARSE ? 0.42 : 0.27);
+    const LaunchPlan plan = make_plan(SPARSE, ELT, BN, OUT_T, OUT_F32, BCOMP, ctx->sm_count,
+                                      ctx->splitk_partials ? ctx->splitk_partial_bytes : 0, p.M, p.N, p.K);
+    pp.group_m = plan.group_m;
     pp.splits = plan.splits;
     pp.split_from = plan.split_from;
     pp.partials = ctx->splitk_partials;
@@ -1113,11 +1130,11 @@ int g_force_splits = 0;   // test hook: 0 = automatic split-K factor
 // partial wave (all of them when there are fewer tiles than pairs, as for the weight gradient of a
 // GPT-2-sized layer: 36 tiles, 74 pairs) are cut into `splits` K ranges so that the wave takes 1/splits
 // of a tile time.  `align` = stages per metadata group (K ranges must start on a group boundary).
-SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int align, int bn, double stage_us)
+SplitPlan pick_split_plan(int sm_count, size_t partial_bytes, int tiles, int k_blocks, int align, int bn, double stage_us)
 {
     SplitPlan none{1, tiles};
-    if (!ctx->splitk_partials) return none;
-    const int pairs = ctx->sm_count / 2;
+    if (partial_bytes == 0) return none;
+    const int pairs = sm_count / 2;
     const int whole = (tiles / pairs) * pairs;
     const int tail = tiles - whole;
     if (tail == 0) return none;
@@ -1126,7 +1143,7 @@ SplitPlan pick_split_plan(const sste_ctx *ctx, int tiles, int k_blocks, int alig
     double best_cost = tile_us;        // time of the last wave, microseconds
     for (int s = 2; s <= 4; ++s) {
         if (k_blocks % (s * align) != 0 || k_blocks / s < 8) continue;
-        if (static_cast<size_t>(tail) * 2 * s * BM * bn * sizeof(float) > ctx->splitk_partial_bytes) continue;
+        if (static_cast<size_t>(tail) * 2 * s * BM * bn * sizeof(float) > partial_bytes) continue;
         if (g_force_splits == s) return SplitPlan{s, whole};
         const int waves = (tail * s + pairs - 1) / pairs;
         // + the second pass (a launch of its own) and the partial tiles' round trip through L2
@@ -1217,6 +1234,37 @@ extern "C" sste_status sste_debug_force_splits(int splits)
 {
     if (splits < 0 || splits > 4) return SSTE_ERR_INVALID_ARG;
     g_force_splits = splits;
+    return SSTE_OK;
+}
+extern "C" sste_status sste_debug_plan(int product, sste_dtype opdt, int O, int I, int T, int sm_count,
+                                       size_t workspace_bytes, int *tile_width, int *splits, int *split_from,
+                                       int *group_m)
+{
+    int elt;
+    uint32_t code;
+    if (!fmt_code(opdt, &elt, &code) || product < 0 || product > 2 || sm_count < 2) return SSTE_ERR_INVALID_ARG;
+    if (!sste_mult128(T) || !sste_mult128(O) || !sste_mult128(I)) return SSTE_ERR_SHAPE;
+    // the (M, N, K) of the launch, as in the three entry points below
+    const int M = product == 2 ? T : O, N = product == 0 ? T : I, K = product == 0 ? I : product == 1 ? T : O;
+    const bool sparse = product != 2, mn = product != 0, out_t = product == 0;
+    int bn = pick_bn(!mn, elt, M, N, K, sm_count / 2);
+    const int cands[4] = {256, (mn && elt == 1) ? 0 : 128, mn ? 0 : 192, (!mn && sparse) ? 224 : 0};
+    for (int c : cands)
+        if (c && c == g_force_bn) bn = c;
+    const size_t partial_bytes =
+        workspace_bytes > SSTE_WS_SPLITK_PARTIALS_OFF + (size_t(1) << 20) ? workspace_bytes - SSTE_WS_SPLITK_PARTIALS_OFF : 0;
+    const LaunchPlan plan = make_plan(sparse, elt, bn, out_t, false, false, sm_count, partial_bytes, M, N, K);
+    if (tile_width) *tile_width = bn;
+    if (splits) *splits = plan.splits;
+    if (split_from) *split_from = plan.split_from;
+    if (group_m) *group_m = plan.group_m;
+    return SSTE_OK;
+}
+extern "C" sste_status sste_debug_tile_coords(int tile, int m_tiles, int n_tiles, int group_m, int *mt, int *nt)
+{
+    if (tile < 0 || m_tiles <= 0 || n_tiles <= 0 || group_m <= 0 || tile >= m_tiles * n_tiles || !mt || !nt)
+        return SSTE_ERR_INVALID_ARG;
+    tile_coords(tile, m_tiles, n_tiles, group_m < m_tiles ? group_m : m_tiles, *mt, *nt);
     return SSTE_OK;
 }
 extern "C" sste_status sste_debug_force_tile_order(int group_m)
