@@ -336,6 +336,14 @@ sste_status sste_debug_force_splits(int splits);
  * plain column-major order) so that tests can cover every order. */
 sste_status sste_debug_force_tile_order(int group_m);
 
+/* The MVUE rule of sste_mvue_sparsify on explicit groups and explicit uniforms, for tests that must reach the cases
+ * a random draw almost never produces (u = 1 - 2^-24, sums that round onto a sampling point, zero magnitudes).
+ * a: device, n groups of four bf16 values; k24: device, n uint32 whose low 24 bits k give u = k * 2^-24;
+ * pos_out: device uint32 [n], q0 | q1 << 2 with q0 < q1 the kept positions; val_out: device float [n][2], the two
+ * kept values in fp32 before any cast. */
+sste_status sste_debug_mvue_groups(sste_ctx *ctx, const void *a, const void *k24, size_t n, void *pos_out,
+                                   void *val_out, void *stream);
+
 /* What the library would decide for a product launch, computed on the host (no device is touched): product 0 =
  * sste_linear_fwd, 1 = sste_linear_bwd_weight, 2 = sste_linear_bwd_input (dense operand), operands of dtype opdt,
  * bf16 output, on a GPU of sm_count SMs with a context workspace of workspace_bytes.  Outputs (each nullable): the

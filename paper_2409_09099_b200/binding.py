@@ -32,6 +32,7 @@ EXPORTS = [
     "sste_project_compress_variant", "sste_beta_init_l1", "sste_srste_decay", "sste_project_amax",
     "sste_decompress", "sste_padded_dim", "sste_pad_2d", "sste_crop_2d", "sste_debug_inject_stall",
     "sste_debug_force_tile_order", "sste_debug_plan", "sste_debug_tile_coords",
+    "sste_debug_mvue_groups",
 ]
 
 
@@ -247,6 +248,11 @@ class Context:
 
     def meta_to_canonical(self, meta, rows, k, dt, out):
         self._check(self.lib.sste_meta_to_canonical(self.handle, _ptr(meta), rows, k, dt, _ptr(out), _stream()))
+
+    def debug_mvue_groups(self, a, k24, pos_out, val_out):
+        """sste_debug_mvue_groups: the MVUE group rule on explicit groups a [n, 4] (bf16) and 24-bit uniforms k24 [n]."""
+        self._check(self.lib.sste_debug_mvue_groups(self.handle, _ptr(a), _ptr(k24), ctypes.c_size_t(a.shape[0]),
+                                                    _ptr(pos_out), _ptr(val_out), _stream()))
 
     def debug_force_splits(self, splits: int):
         self._check(self.lib.sste_debug_force_splits(splits))

@@ -273,7 +273,8 @@ struct MvueGroup {
 // Inclusion probabilities p_i = min(1, c |a_i|) with sum 2, kept values a_i / p_i, systematic sampling
 // with one uniform u.  With x the first largest magnitude and rest the sum of the others:
 //   clipped   (m_x >= rest): x is kept as is; one other element j, chosen with probability m_j / rest
-//                            by the point u*rest on the others' cumulative sums, carries sign(a_j)*rest;
+//                            by the point u*rest on the others' cumulative sums (kept below rest), carries
+//                            sign(a_j)*rest;
 //   unclipped (m_x <  rest): the points u*S/2 and u*S/2 + S/2 on the cumulative sums pick two elements,
 //                            both carry sign(a_j)*S/2.
 // The kernel is bound by instruction issue, not by HBM, so this is written for instruction count: no
@@ -304,8 +305,12 @@ __device__ __forceinline__ MvueGroup mvue_group(uint32_t p01, uint32_t p23, floa
     const float c0 = clipped ? z0 : m0, c1 = clipped ? z1 : s1, c2 = clipped ? z2 : s2;
     const float r1 = __fmul_rn(u, h);
     const float r2 = __fadd_rn(r1, h);
+    // Clipped: a point that rounding put AT rest (possible only when u * rest is subnormal) counts as just below
+    // it, which selects the last other element of nonzero magnitude.  (rest == 0: the second operand is a NaN and
+    // fminf returns r1; that case is decided below.)
+    const float r1c = clipped ? fminf(r1, __uint_as_float(__float_as_uint(rest) - 1u)) : r1;
     // number of cumulative sums at or below each point: compares as 0 / -1, one three-input add each
-    const int j1 = -(fset_le(c0, r1) + fset_le(c1, r1) + fset_le(c2, r1));
+    const int j1 = -(fset_le(c0, r1c) + fset_le(c1, r1c) + fset_le(c2, r1c));
     const int n2 = -(fset_le(c0, r2) + fset_le(c1, r2) + fset_le(c2, r2));
     // index pair before ordering: (other, x) when clipped; (j1, j2) otherwise, where a first point in the
     // last element (j1 = 3) gives the pair (2, 3)
@@ -329,6 +334,24 @@ __device__ __forceinline__ MvueGroup mvue_group(uint32_t p01, uint32_t p23, floa
     r.v0 = swap ? vb : va;
     r.v1 = swap ? va : vb;
     return r;
+}
+
+// The group rule on explicit inputs (test / debug): group i = four bf16 values a[4 i .. 4 i + 3] and the uniform
+// u[i] = k[i] * 2^-24; out: kept positions (q0 | q1 << 2) and the two fp32 values before the cast.
+__global__ void __launch_bounds__(EW_THREADS)
+mvue_groups_kernel(const uint2 *__restrict__ a, const uint32_t *__restrict__ k24, size_t n, uint32_t *__restrict__ pos,
+                   float2 *__restrict__ val)
+{
+    sste_pdl_trigger();
+    sste_pdl_wait();
+    for (size_t i = static_cast<size_t>(blockIdx.x) * EW_THREADS + threadIdx.x; i < n;
+         i += static_cast<size_t>(gridDim.x) * EW_THREADS) {
+        const uint2 g = a[i];
+        const float u = __uint2float_rn(k24[i] & 0xffffffu) * 0x1p-24f;
+        const MvueGroup r = mvue_group(g.x, g.y, u);
+        pos[i] = r.q0 | (r.q1 << 2);
+        val[i] = make_float2(r.v0, r.v1);
+    }
 }
 
 // ---------------------------------------------------------------- MVUE + compress (transposing)
@@ -1046,5 +1069,19 @@ extern "C" sste_status sste_crop_2d(sste_ctx *ctx, const void *src, int rows_p, 
     const size_t n = static_cast<size_t>(rows) * cols;
     sste_launch(crop_2d_kernel, dim3(grid_for(n, ctx->sm_count)), dim3(EW_THREADS), 0, static_cast<cudaStream_t>(stream),
                 static_cast<const uint16_t *>(src), cols_p, static_cast<uint16_t *>(dst), cols, n);
+    return launch_result();
+}
+
+extern "C" sste_status sste_debug_mvue_groups(sste_ctx *ctx, const void *a, const void *k24, size_t n, void *pos_out,
+                                              void *val_out, void *stream)
+{
+    if (!ctx || !a || !k24 || !pos_out || !val_out || n == 0) return SSTE_ERR_INVALID_ARG;
+    if (!sste_aligned(a, 8) || !sste_aligned(k24, 4) || !sste_aligned(pos_out, 4) || !sste_aligned(val_out, 8))
+        return SSTE_ERR_ALIGN;
+    sste_device_guard guard(ctx->device);
+    if (!guard.ok) return SSTE_ERR_CUDA;
+    sste_launch(mvue_groups_kernel, dim3(grid_for(n, ctx->sm_count)), dim3(EW_THREADS), 0, static_cast<cudaStream_t>(stream),
+                static_cast<const uint2 *>(a), static_cast<const uint32_t *>(k24), n, static_cast<uint32_t *>(pos_out),
+                static_cast<float2 *>(val_out));
     return launch_result();
 }
