@@ -358,3 +358,33 @@ def test_tile_order_does_not_change_the_products(ctx, group_m):
     for a, ref in zip(results[2, group_m][:3], refs):
         assert rel_fro(a.float().cpu().numpy(), ref) <= BF16_GEMM_TOL
     assert ctx.poll_device_status() == 0
+
+
+@pytest.mark.parametrize("fp8", [False, True])
+def test_projection_on_every_group_over_an_alphabet(ctx, fp8):
+    """All 12^4 groups over an alphabet with zeros, -0, subnormals, adjacent bf16 values, ties and huge ratios:
+    values, metadata and dense copy bit for bit (bf16 and E4M3), and the beta reduction on the same tensor."""
+    from paper_2409_09099_b200 import binding as B
+    alphabet = np.array([0.0, -0.0, 1.0, -1.0, 1.0078125, 2.0, -3.0, 0.5, 2.0 ** -17, 2.0 ** -126, -(2.0 ** -133), 65280.0],
+                        dtype=np.float32)
+    idx = np.stack(np.meshgrid(*[np.arange(len(alphabet))] * 4, indexing="ij"), -1).reshape(-1, 4)
+    flat = np.zeros(128 * 768, np.float32)
+    flat[: idx.size] = alphabet[idx].reshape(-1)
+    W = synth.to_bf16_bits(flat.reshape(128, 768))
+    O, I = W.shape
+    beta32, w_amax = np.float32(1.4837), np.float32(65280.0 * 1.4837)
+    dt, odt = (B.E4M3, orc.E4M3) if fp8 else (B.BF16, orc.BF16)
+    vals, meta = ctx.alloc_compressed(O, I, dt)
+    dense = torch.empty((O, I), dtype=B._TORCH_DT[dt], device=DEV)
+    beta = torch.full((1,), float(beta32), dtype=torch.float32, device=DEV)
+    amax = torch.full((1,), float(w_amax), dtype=torch.float32, device=DEV)
+    ctx.project_compress(dbf16(W), beta, vals, meta, dense, w_amax_dev=amax if fp8 else None)
+    ov, om, od = orc.project_compress(W, beta32, odt=odt, wscale=orc.fp8_scale(w_amax, orc.E4M3) if fp8 else 1.0)
+    bits = (lambda t: t.view(torch.uint8).cpu().numpy()) if fp8 else bits16
+    assert np.array_equal(bits(vals), ov)
+    assert np.array_equal(bits(dense), od)
+    assert np.array_equal(canonical_meta(ctx, meta, O, I, dt), om)
+    got = torch.zeros(1, dtype=torch.float32, device=DEV)
+    ctx.beta_init(dbf16(W), got)
+    ref = orc.beta(W)[0]
+    assert abs(got.item() - ref) <= 1e-6 * abs(ref)
