@@ -580,7 +580,10 @@ def run_gpu(args):
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     if world > 1:
-        os.environ.setdefault("NCCL_DEBUG", "WARN")
+        # the communicator log (rings / trees, NVLS or not) goes to stderr; stdout carries the one JSON line
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT,GRAPH")
+        os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
         dist.init_process_group("nccl", device_id=torch.device(dev))
     sampler = ClockSampler(local_rank)
     sampler.start()
