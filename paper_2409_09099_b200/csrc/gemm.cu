@@ -11,8 +11,12 @@
 //   warp 0    TMA producer (both CTAs; all transaction bytes land on the leader's barrier)
 //   warp 1    leader CTA: tcgen05.mma[.sp] issue; both CTAs: tensor-memory allocation
 //   warps 2-5 epilogue: TMEM -> registers -> bf16 -> shared memory -> TMA store
-//   warps 6-9 (sparse only) metadata: HBM -> registers -> tensor memory (tcgen05.st), so that no
-//             metadata copy sits between two MMAs in the tensor pipe (a tcgen05.cp there drains it)
+//   warps 6-9 sparse A: metadata HBM -> registers -> tensor memory (tcgen05.st), so that no
+//             metadata copy sits between two MMAs in the tensor pipe (a tcgen05.cp there drains it);
+//             compressed B (grad_X from the forward's operand): expansion of values + metadata
+//             into the dense shared-memory stage
+// Output tiles are handed out band by band (tile_coords) so that operands are read from HBM about
+// once; tile width, split-K plan and band height come from cost models on the host (make_plan).
 // Every wait is bounded: on expiry the CTA records SSTE_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 
