@@ -193,7 +193,7 @@ def run_reference(args):
 
 
 def workload_config(cfg_id, cfg, n_gpus):
-    return {"workload": f"BASELINE config {cfg_id}: " + ", ".join(f"{L.name} W[{L.O},{L.I}] x {L.T} tokens" for L in cfg["layers"]),
+    return {"workload": f"config {cfg_id}: " + ", ".join(f"{L.name} W[{L.O},{L.I}] x {L.T} tokens" for L in cfg["layers"]),
             "precision": "fp8 (e4m3 fwd / e5m2 bwd)" if cfg["fp8"] else "bf16",
             "tokens_per_gpu": cfg["layers"][0].T, "parallelism": f"dp{n_gpus} (token shards; grad_W all-reduced over NCCL when n_gpus > 1)",
             "l2": "flushed between timed steps (512 MiB write)", "launch": "n_gpus = 1: one CUDA-graph replay per step, grad_W on a side stream beside grad_X "
@@ -660,7 +660,7 @@ def run_model(args):
     line = {"metric": METRIC, "value": model.flops_per_step() / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "BASELINE config 4: 12-layer GPT-2-124M-shaped decoder, 8 x 1024 uniform token ids, all 48 "
+            "config": {"workload": "config 4: 12-layer GPT-2-124M-shaped decoder, 8 x 1024 uniform token ids, all 48 "
                                    "linears through libsste; attention, layer norms, embeddings, loss and AdamW in torch",
                        "note": "value counts the S-STE linears' 6*T*I*O flops over the WHOLE training step"},
             "libsste_fraction_of_step": inside / total, "loss": float(loss), "gpu_launches": int(launches),
@@ -685,7 +685,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=5,
-                    help="BASELINE config id (5 = FP8 7B-shaped FFN, the largest single-GPU workload; 2, 3 bf16)")
+                    help="benchmark config id (5 = FP8 7B-shaped FFN, the largest single-GPU workload; 2, 3 bf16)")
     ap.add_argument("--no-overlap", action="store_true",
                     help="run grad_W and grad_X back to back instead of grad_W on a side stream beside grad_X")
     ap.add_argument("--no-graph", action="store_true", help="launch the timed steps eagerly instead of replaying a CUDA graph")
