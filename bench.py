@@ -543,7 +543,8 @@ def measure_config(cfg_id, args, env, full):
     rooflines = stage_rooflines(cfg, per_call_us, hot_us, peaks, cfg_id)
     stage_us = {st: sum(per_call_step_us.get(l, 0.0) for l in labels) for st, labels in STAGES.items()}
     total_us = sum(stage_us.values()) or 1.0
-    dom = max(stage_us, key=stage_us.get)
+    # the dominant KERNEL: the stage whose main kernel (helpers apart) takes the most time per step
+    dom = max(STAGES, key=lambda st: per_call_step_us.get(STAGES[st][-1], 0.0))
     breakdown = {st: {"ms_per_step": stage_us[st] * 1e-3, "share": stage_us[st] / total_us,
                       "roofline_frac": rooflines[st]["frac"], "bound": rooflines[st]["bound"]} for st in STAGES}
     rep_ms = [r / steps for r in per_rep]
