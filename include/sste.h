@@ -353,6 +353,10 @@ sste_status sste_debug_plan(int product, sste_dtype opdt, int O, int I, int T, i
                             int *tile_width, int *splits, int *split_from, int *group_m);
 sste_status sste_debug_tile_coords(int tile, int m_tiles, int n_tiles, int group_m, int *mt, int *nt);
 
+/* Host-only self-check of the once-per-device bookkeeping behind per-device kernel attributes (a context may live on
+ * any device ordinal, and the opt-in to large dynamic shared memory is per device).  SSTE_OK if it behaves. */
+sste_status sste_debug_selftest_device_once(void);
+
 /* Test hook for the bounded waits.  While armed (on != 0), a dense sste_linear_bwd_input (Wt_dense given, bf16
  * output) whose output is ONE tile (T <= 256, I <= 256) leaves the last K stage of its operand pipeline unloaded
  * and limits every device-side wait to one millisecond instead of two seconds: the wait for that stage runs out,

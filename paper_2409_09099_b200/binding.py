@@ -32,7 +32,7 @@ EXPORTS = [
     "sste_project_compress_variant", "sste_beta_init_l1", "sste_srste_decay", "sste_project_amax",
     "sste_decompress", "sste_padded_dim", "sste_pad_2d", "sste_crop_2d", "sste_debug_inject_stall",
     "sste_debug_force_tile_order", "sste_debug_plan", "sste_debug_tile_coords",
-    "sste_debug_mvue_groups",
+    "sste_debug_mvue_groups", "sste_debug_selftest_device_once",
 ]
 
 

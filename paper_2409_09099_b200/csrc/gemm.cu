@@ -1264,6 +1264,25 @@ extern "C" sste_status sste_debug_plan(int product, sste_dtype opdt, int O, int 
     if (group_m) *group_m = plan.group_m;
     return SSTE_OK;
 }
+// Host-only self-check of the once-per-device guard the launches use for per-device kernel attributes: `fn` must
+// run once per device ordinal, again after a failure, and never for a device that already succeeded.
+extern "C" sste_status sste_debug_selftest_device_once(void)
+{
+    DeviceOnce once;
+    int calls[4] = {0, 0, 0, 0};
+    bool fail_next = true;
+    auto fn = [&](int dev) {
+        return once.run(dev, [&] {
+            ++calls[dev];
+            if (dev == 2 && fail_next) { fail_next = false; return false; }   // first attempt on device 2 fails
+            return true;
+        });
+    };
+    const bool r0 = fn(0), r0b = fn(0), r1 = fn(1), r2 = fn(2), r2b = fn(2), r2c = fn(2), r3 = fn(3), r1b = fn(1);
+    const bool ok = r0 && r0b && r1 && !r2 && r2b && r2c && r3 && r1b && calls[0] == 1 && calls[1] == 1 &&
+                    calls[2] == 2 && calls[3] == 1;
+    return ok ? SSTE_OK : SSTE_ERR_INVALID_ARG;
+}
 extern "C" sste_status sste_debug_tile_coords(int tile, int m_tiles, int n_tiles, int group_m, int *mt, int *nt)
 {
     if (tile < 0 || m_tiles <= 0 || n_tiles <= 0 || group_m <= 0 || tile >= m_tiles * n_tiles || !mt || !nt)

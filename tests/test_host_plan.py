@@ -81,3 +81,8 @@ def test_plan_rejects_bad_arguments(lib):
     assert lib.sste_debug_plan(0, B.F32, 128, 128, 128, 148, ctypes.c_size_t(0), None, None, None, None) == B.ERR_INVALID_ARG
     assert lib.sste_debug_plan(0, B.BF16, 100, 128, 128, 148, ctypes.c_size_t(0), None, None, None, None) == B.ERR_SHAPE
     assert lib.sste_debug_plan(0, B.BF16, 128, 128, 128, 148, ctypes.c_size_t(0), None, None, None, None) == B.OK
+
+
+def test_per_device_attribute_guard(lib):
+    """The launches set a kernel's shared-memory opt-in once per device ordinal (and retry after a failure)."""
+    assert lib.sste_debug_selftest_device_once() == B.OK
